@@ -1,0 +1,150 @@
+/*
+ * libape -- APE (Adaptive Parallel Encoding, arxiv 2502.05431) attention for NVIDIA B200 (sm_100a).
+ *
+ * C ABI: plain pointers and sizes only.  Unless said otherwise a pointer is a DEVICE pointer that the
+ * caller owns; arrays of descriptors (requests, spans) are HOST arrays that are read during the call and
+ * may be freed as soon as it returns.  Every function returns APE_OK (0) or a negative ape_status code;
+ * nothing throws, aborts, traps or prints.  All tensors are bf16 with the head dimension contiguous;
+ * strides are in ELEMENTS.
+ *
+ * Data model (paper, section "Parallel Encoding": a query is augmented by a subset of independently
+ * pre-cached contexts; section "Prepending Shared Prefix": one shared prefix in front of all of them):
+ *   - one KV pool  K, V : [n_tokens, H_kv, d]  holds every cached token of every request;
+ *   - the shared prefix, each cached context C_i and the query's own K/V are SPANS (start, len) of pool
+ *     tokens.  Contexts are addressed through the span table only, never re-packed, so inserting,
+ *     removing or re-ordering contexts is an edit of that table;
+ *   - query rows Q and outputs O : [rows, H_q, d]; consecutive query heads share a KV head
+ *     (g = h / (H_q / H_kv)).
+ *
+ * Two operations, each split into a plan (host work: validation, tile lists, upload; may block) and
+ * a launch (asynchronous on the caller's stream, no allocation, no host synchronisation):
+ *
+ *   ape_attend           Eq. 5 of the paper (section "Formulation"): softmax attention of the query rows over
+ *                        [prefix | all contexts | causal query segment] in which context logits are
+ *                        divided by the temperature T and the summed context weight Z_C enters as Z_C^S.
+ *   ape_encode_contexts  the pre-caching attention (section "Parallel Encoding", first step): every
+ *                        context row attends to the whole prefix and causally to its own context only.
+ */
+#ifndef APE_H_
+#define APE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ape_handle_s *ape_handle_t;
+typedef struct ape_plan_s *ape_plan_t;
+
+enum ape_status {
+    APE_OK = 0,
+    APE_ERR_INVALID_ARG = -1, /* null pointer, negative count, span outside the pool, len < q_len ...      */
+    APE_ERR_SHAPE = -2,       /* H_q % H_kv != 0, H_q/H_kv not a power of two <= 16, head_dim not 64 or 128 */
+    APE_ERR_ALIGN = -3,       /* pointer not 16-byte aligned or stride not a multiple of 8 elements        */
+    APE_ERR_RANGE = -4,       /* T or S not finite and > 0, kv_extra outside the reserved capacity         */
+    APE_ERR_LAYOUT = -5,      /* a tensor cannot be described to the copy engine (extent over 2^31 ...)     */
+    APE_ERR_WORKSPACE = -6,   /* workspace missing, misaligned (256 B) or too small                        */
+    APE_ERR_CUDA = -7,        /* a CUDA runtime or driver call failed                                      */
+    APE_ERR_TIMEOUT = -8,     /* a kernel gave up on a bounded wait (reported by ape_get_status)           */
+    APE_ERR_NOMEM = -9,       /* host or device allocation failed while planning                           */
+    APE_ERR_MODE = -10        /* plan used with the wrong entry point                                      */
+};
+
+typedef enum { APE_PREFILL = 0, APE_DECODE = 1 } ape_mode_t;
+
+typedef struct {
+    int32_t n_q_heads;   /* H_q                                                  */
+    int32_t n_kv_heads;  /* H_kv, divides H_q; H_q/H_kv a power of two <= 16     */
+    int32_t head_dim;    /* d: 64 or 128                                         */
+    float softmax_scale; /* logit scale c; 0 selects 1/sqrt(d) (Eq. 1)           */
+} ape_shape_t;
+
+typedef struct { int64_t start, len; } ape_span_t;        /* tokens of the KV pool, len >= 0 */
+
+typedef struct {          /* K and V share geometry: element (t, g, e) at base[t*token_stride + g*head_stride + e] */
+    const void *k, *v;
+    int64_t n_tokens, token_stride, head_stride;
+} ape_kv_pool_t;
+
+typedef struct {          /* Q or O rows: element (r, h, e) at data[r*token_stride + h*head_stride + e] */
+    void *data;
+    int64_t n_rows, token_stride, head_stride;
+} ape_rows_t;
+
+typedef struct {          /* one request (HOST struct; ctx is a HOST array) */
+    int64_t q_start, q_len;        /* its rows of Q and O; q_len >= 1 (decode: q_len == 1)                     */
+    ape_span_t prefix;             /* shared prefix P, len may be 0                                            */
+    const ape_span_t *ctx;         /* the N cached contexts C_1..C_N in any order; entries may be empty        */
+    int32_t n_ctx;                 /* N >= 0                                                                   */
+    ape_span_t query_kv;           /* the query segment's own K/V, len l_k >= q_len; row i sees keys            */
+                                   /* j <= i + (l_k - q_len) (causal, aligned to the end)                      */
+    int64_t query_kv_capacity;     /* >= query_kv.len: pool tokens reserved from query_kv.start for appends    */
+} ape_request_t;
+
+/* Library instance bound to one device.  Allocates a 4-byte device status word.  `device` is a CUDA ordinal. */
+int ape_create(ape_handle_t *handle, int device);
+int ape_destroy(ape_handle_t handle);
+
+/*
+ * Plan an attend over n_req independent requests that share one pool and one Q / O tensor.
+ * mode APE_PREFILL: tensor-core kernel for q_len rows per request.  mode APE_DECODE: q_len must be 1;
+ * split-KV streaming kernel.  `lse` (nullable, device, fp32 [q rows, H_q]) receives the natural log of
+ * Eq. 5's denominator.  Builds tile lists and work assignments, uploads them (cudaMalloc + blocking copy).
+ * The plan keeps the device pointers given here; their contents may change between launches.
+ */
+int ape_attend_plan(ape_handle_t handle, const ape_shape_t *shape, const ape_kv_pool_t *pool,
+                    const ape_rows_t *q, const ape_rows_t *out, float *lse,
+                    const ape_request_t *requests, int32_t n_req, ape_mode_t mode, ape_plan_t *plan);
+
+/*
+ * Plan the block-diagonal encoding of n_ctx contexts against one shared prefix.  `q` and `out` are aligned
+ * with the pool: row t belongs to pool token t (only rows inside the context spans are read / written).
+ * `lse` (nullable, fp32 [pool rows, H_q]) receives each row's log-sum-exp.
+ */
+int ape_encode_plan(ape_handle_t handle, const ape_shape_t *shape, const ape_kv_pool_t *pool,
+                    const ape_rows_t *q, const ape_rows_t *out, float *lse,
+                    const ape_span_t *prefix, const ape_span_t *ctx, int32_t n_ctx, ape_plan_t *plan);
+
+/* Bytes of device scratch a launch of this plan needs (a multiple of 256; may be 0). */
+int ape_plan_workspace_bytes(ape_plan_t plan, size_t *bytes);
+int ape_plan_destroy(ape_plan_t plan);
+
+/*
+ * Launch APE attention (Eq. 5; the two-accumulator + log-sum-exp merge of the appendix "Efficient
+ * Implementation").  T: attention temperature, S: scaling factor (the exponent of the context mass in
+ * Eq. 5; a caller who tuned with the paper's S*T parametrisation passes that product).  Both finite, > 0.
+ * kv_extra: tokens appended to every request's query segment since planning (decode step t passes t;
+ * 0 <= kv_extra <= capacity - len; prefill plans require 0).  `workspace`: device, 256-byte aligned,
+ * at least ape_plan_workspace_bytes; contents undefined afterwards.  `stream`: a cudaStream_t (0 = default).
+ * Asynchronous; launches that share a workspace must be stream-ordered.
+ */
+int ape_attend(ape_plan_t plan, float T, float S, int64_t kv_extra,
+               void *workspace, size_t workspace_bytes, void *stream);
+
+/* Launch the context pre-encoding attention of an encode plan.  No T, no S (they apply to queries only). */
+int ape_encode_contexts(ape_plan_t plan, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * End-to-end variant for callers whose tensors live in HOST memory: copies h_q (the Q tensor) and the
+ * K / V pools host-to-device into the plan's device buffers, launches ape_attend, copies O back to h_out,
+ * all on `stream`, then synchronises the stream.  Host buffers have the same geometry as the device
+ * tensors (dense: token_stride = heads * d, head_stride = d) and should be pinned.
+ * *h2d_bytes / *d2h_bytes (nullable) receive the bytes moved.
+ */
+int ape_attend_host(ape_plan_t plan, float T, float S, int64_t kv_extra, void *workspace, size_t workspace_bytes,
+                    const void *h_q, const void *h_k_pool, const void *h_v_pool, void *h_out,
+                    size_t *h2d_bytes, size_t *d2h_bytes, void *stream);
+
+/* Kernels launched by the last ape_attend / ape_encode_contexts call on this plan. */
+int ape_plan_last_launches(ape_plan_t plan, int32_t *n_launches);
+
+/* Synchronises the device and returns the device status word (0, or APE_ERR_TIMEOUT) in *device_status; clears it. */
+int ape_get_status(ape_handle_t handle, int32_t *device_status);
+const char *ape_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* APE_H_ */
