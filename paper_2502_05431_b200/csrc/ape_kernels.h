@@ -1,0 +1,76 @@
+// Internal launch interface between the host API (ape_api.cu) and the kernels.
+#pragma once
+
+#include "ape_common.cuh"
+
+namespace ape {
+
+constexpr int kDecodeTile = 64;     // tokens per pipeline stage of the decode kernel
+constexpr int kAttnTileN = 128;     // keys per tile of the tensor-core (prefill / encode) kernel
+constexpr int kAttnRows = 256;      // packed (token, head-in-group) rows per row block of that kernel (two 128-row halves)
+
+struct DecodeParams {
+    const DevTile* tiles;
+    const DevItem* items;
+    const int32_t* cta_item_begin;   // [n_cta + 1]
+    const DevReq* reqs;
+    RowsDesc q;
+    float* ws_o;                     // [n_slots][G][D]  unnormalised partial outputs
+    float* ws_ml;                    // [n_slots][G][2]  running maximum (base-2 logits) and sum
+    float scale_oth_log2;            // c * log2(e)
+    float scale_ctx_log2;            // c / T * log2(e)
+    int32_t kv_extra;
+    int32_t G;
+    int32_t n_stages;
+    int* status;
+};
+
+size_t decode_smem_bytes(int D, int G, int n_stages);
+int decode_pick_stages(int D, int G, size_t smem_limit);
+cudaError_t decode_set_smem_attr(int D, size_t smem_bytes);
+cudaError_t launch_decode(int D, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const DecodeParams& p,
+                          int n_cta, size_t smem_bytes, cudaStream_t stream);
+
+// Tensor-core attention kernel shared by query prefill and context encoding.
+struct AttnParams {
+    const DevTile* tiles;
+    const DevItem* items;
+    const int32_t* cta_item_begin;   // [n_groups + 1]; CTA b serves group b / n_sib as sibling b % n_sib
+    const DevReq* reqs;
+    RowsDesc out;                    // SEG_FINAL items write here
+    float* lse_out;                  // nullable, [rows, H_q] natural-log LSE for SEG_FINAL items
+    float* ws_o;                     // [n_slots][kAttnRows][D]
+    float* ws_ml;                    // [n_slots][kAttnRows][2]
+    float scale_oth_log2;
+    float scale_ctx_log2;
+    int32_t G;
+    int32_t H_q;
+    int32_t n_sib;                   // sibling CTAs per group (row blocks that stream the same tiles together)
+    int32_t q_rows_are_pool;         // encode: Q / O rows are pool tokens (row = context start + i)
+    int* status;
+};
+
+size_t attn_smem_bytes(int D);
+cudaError_t attn_set_smem_attr(int D, size_t smem_bytes);
+cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                        const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream);
+
+// Merge of the partials: hierarchical softmax identity inside each segment, then Eq. 5's scaling factor.
+struct MergeParams {
+    const DevMerge* groups;
+    const DevReq* reqs;
+    int32_t n_groups;
+    int32_t rows_per_slot;           // G (decode) or kAttnRows (prefill)
+    int32_t tokens_per_block;        // query tokens per row block: rows_per_slot / G
+    const float* ws_o;
+    const float* ws_ml;
+    RowsDesc out;
+    float* lse_out;                  // nullable, [rows, H_q]
+    float S;
+    int32_t G;
+    int32_t H_q;
+    int32_t D;
+};
+cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
+
+}  // namespace ape

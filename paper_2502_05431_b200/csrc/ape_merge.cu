@@ -1,0 +1,100 @@
+// Merge kernel: turns the per-item partials (m, l, O~), kept in base-2 units, into the final output.
+//   1. inside each segment (context / non-context) the partials of all splits are combined by the
+//      hierarchical softmax identity (appendix "Hierarchical Formula for Softmax Attention"):
+//      LSE = logsumexp_s(m_s + log2 l_s),  O = sum_s 2^(LSE_s - LSE) O_s;
+//   2. the context log-sum-exp is multiplied by the scaling factor S and the two segments are merged by a
+//      softmax over [S * LSE_C, LSE_other] (Eq. 5; appendix "Efficient Implementation").
+// One warp per output row (query token, query head); lanes cover the head dimension.
+#include "ape_common.cuh"
+#include "ape_kernels.h"
+
+namespace ape {
+
+namespace {
+
+constexpr float kLn2 = 0.6931471805599453f;
+
+template <int VEC>
+__device__ __forceinline__ void combine_segment(const float* __restrict__ ws_o, const float* __restrict__ ws_ml,
+                                                int slot0, int n, int stride, int rows_per_slot, int row, int D,
+                                                int lane, float& M, float& L, float (&acc)[VEC])
+{
+    M = -INFINITY; L = 0.f;
+    #pragma unroll
+    for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
+    for (int i = 0; i < n; ++i) {
+        const size_t slot = static_cast<size_t>(slot0) + static_cast<size_t>(i) * stride;
+        const float2 ml = *reinterpret_cast<const float2*>(ws_ml + (slot * rows_per_slot + row) * 2);
+        if (!(ml.y > 0.f)) continue;                 // empty partial
+        const float Mn = fmaxf(M, ml.x);
+        const float f_old = fast_exp2(M - Mn), f_new = fast_exp2(ml.x - Mn);
+        const float* src = ws_o + (slot * rows_per_slot + row) * D + lane * VEC;
+        float x[VEC];
+        if constexpr (VEC == 4) { const float4 t = *reinterpret_cast<const float4*>(src); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
+        else { const float2 t = *reinterpret_cast<const float2*>(src); x[0] = t.x; x[1] = t.y; }
+        #pragma unroll
+        for (int v = 0; v < VEC; ++v) acc[v] = acc[v] * f_old + x[v] * f_new;
+        L = L * f_old + ml.y * f_new;
+        M = Mn;
+    }
+}
+
+template <int VEC>
+__global__ void __launch_bounds__(256) ape_merge_kernel(const MergeParams p)
+{
+    const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    const int group = warp_global / p.rows_per_slot;
+    const int row = warp_global - group * p.rows_per_slot;
+    if (group >= p.n_groups) return;
+    const DevMerge g = p.groups[group];
+    const DevReq rq = p.reqs[g.req];
+    const int tok = g.row_block * p.tokens_per_block + row / p.G;     // query row inside the request
+    const int hg = row % p.G;
+    if (tok >= rq.q_len) return;
+
+    float Mc, Lc, Mo, Lo, ac[VEC], ao[VEC];
+    combine_segment<VEC>(p.ws_o, p.ws_ml, g.ctx_slot0, g.ctx_n, g.slot_stride, p.rows_per_slot, row, p.D, lane, Mc, Lc, ac);
+    combine_segment<VEC>(p.ws_o, p.ws_ml, g.oth_slot0, g.oth_n, g.slot_stride, p.rows_per_slot, row, p.D, lane, Mo, Lo, ao);
+
+    // base-2 log-sum-exps of the two segments; the context one is multiplied by S (Eq. 5: Z_C^S)
+    const float lse_c = (Lc > 0.f) ? p.S * (Mc + fast_log2(Lc)) : -INFINITY;
+    const float lse_o = (Lo > 0.f) ? (Mo + fast_log2(Lo)) : -INFINITY;
+    const float top = fmaxf(lse_c, lse_o);
+    float wc = 0.f, wo = 0.f, lam = -INFINITY;
+    if (top > -INFINITY) {
+        const float ec = fast_exp2(lse_c - top), eo = fast_exp2(lse_o - top);
+        const float inv = 1.f / (ec + eo);
+        wc = (Lc > 0.f) ? ec * inv / Lc : 0.f;        // weight of the context segment over its own normaliser
+        wo = (Lo > 0.f) ? eo * inv / Lo : 0.f;
+        lam = (top + fast_log2(ec + eo)) * kLn2;
+    }
+    const int h = g.kv_head * p.G + hg;
+    __nv_bfloat16* dst = p.out.data + static_cast<int64_t>(rq.q_row0 + tok) * p.out.token_stride
+                         + static_cast<int64_t>(h) * p.out.head_stride + lane * VEC;
+    float r[VEC];
+    #pragma unroll
+    for (int v = 0; v < VEC; ++v) r[v] = wc * ac[v] + wo * ao[v];
+    if constexpr (VEC == 4) {
+        uint2 pk; pk.x = pack_bf16x2(r[0], r[1]); pk.y = pack_bf16x2(r[2], r[3]);
+        *reinterpret_cast<uint2*>(dst) = pk;
+    } else {
+        *reinterpret_cast<uint32_t*>(dst) = pack_bf16x2(r[0], r[1]);
+    }
+    if (p.lse_out != nullptr && lane == 0)
+        p.lse_out[static_cast<int64_t>(rq.q_row0 + tok) * p.H_q + h] = lam;
+}
+
+}  // namespace
+
+cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream)
+{
+    const long long warps = static_cast<long long>(p.n_groups) * p.rows_per_slot;
+    if (warps == 0) return cudaSuccess;
+    const int blocks = static_cast<int>((warps * 32 + 255) / 256);
+    if (p.D == 128) ape_merge_kernel<4><<<blocks, 256, 0, stream>>>(p);
+    else ape_merge_kernel<2><<<blocks, 256, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace ape
