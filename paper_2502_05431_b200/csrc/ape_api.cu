@@ -1,0 +1,573 @@
+// Host side of libape: argument validation, planning (tile lists, work assignment, copy-engine descriptors)
+// and the launches behind the C ABI declared in include/ape.h.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/ape.h"
+#include "ape_kernels.h"
+
+using namespace ape;
+
+namespace {
+
+enum PlanKind { PLAN_PREFILL = 0, PLAN_DECODE = 1, PLAN_ENCODE = 2 };
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+struct ape_handle_s {
+    int device = 0;
+    int n_sm = 0;
+    size_t smem_optin = 0;
+    int* d_status = nullptr;
+    EncodeTiledFn encode_tiled = nullptr;
+};
+
+struct ape_plan_s {
+    ape_handle_t h = nullptr;
+    PlanKind kind = PLAN_PREFILL;
+    ape_shape_t shape{};
+    float c = 0.f;
+    int G = 1;
+    ape_kv_pool_t pool{};
+    ape_rows_t q{}, out{};
+    float* lse = nullptr;
+    // device metadata (one allocation)
+    void* d_blob = nullptr;
+    DevTile* d_tiles = nullptr;
+    DevItem* d_items = nullptr;
+    int32_t* d_cta_begin = nullptr;
+    DevReq* d_reqs = nullptr;
+    DevMerge* d_merge = nullptr;
+    int n_items = 0, n_cta = 0, n_merge = 0, n_sib = 1, n_slots = 0;
+    int n_stages = 0;
+    size_t smem_bytes = 0;
+    size_t ws_bytes = 0;
+    int64_t max_kv_extra = 0;
+    CUtensorMap tm_q{}, tm_k{}, tm_v{};
+    int32_t last_launches = 0;
+};
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(const ape_shape_t* s, int* G_out, float* c_out) {
+    if (!s) return APE_ERR_INVALID_ARG;
+    if (s->n_q_heads <= 0 || s->n_kv_heads <= 0 || s->n_q_heads % s->n_kv_heads) return APE_ERR_SHAPE;
+    const int G = s->n_q_heads / s->n_kv_heads;
+    if (G > 16 || (G & (G - 1))) return APE_ERR_SHAPE;
+    if (s->head_dim != 64 && s->head_dim != 128) return APE_ERR_SHAPE;
+    if (!(s->softmax_scale >= 0.f) || !std::isfinite(s->softmax_scale)) return APE_ERR_RANGE;
+    *G_out = G;
+    *c_out = s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / std::sqrt(static_cast<float>(s->head_dim));
+    return APE_OK;
+}
+
+int check_pool(const ape_kv_pool_t* p, const ape_shape_t* s) {
+    if (!p || !p->k || !p->v || p->n_tokens <= 0) return APE_ERR_INVALID_ARG;
+    if (!aligned16(p->k) || !aligned16(p->v)) return APE_ERR_ALIGN;
+    if (p->head_stride % 8 || p->token_stride % 8) return APE_ERR_ALIGN;
+    if (p->head_stride < s->head_dim || p->token_stride < static_cast<int64_t>(s->n_kv_heads - 1) * p->head_stride + s->head_dim)
+        return APE_ERR_INVALID_ARG;
+    if (p->n_tokens >= (1ll << 31) - 256) return APE_ERR_LAYOUT;
+    return APE_OK;
+}
+
+int check_rows(const ape_rows_t* r, const ape_shape_t* s) {
+    if (!r || !r->data || r->n_rows <= 0) return APE_ERR_INVALID_ARG;
+    if (!aligned16(r->data)) return APE_ERR_ALIGN;
+    if (r->head_stride % 8 || r->token_stride % 8) return APE_ERR_ALIGN;
+    if (r->head_stride < s->head_dim || r->token_stride < static_cast<int64_t>(s->n_q_heads - 1) * r->head_stride + s->head_dim)
+        return APE_ERR_INVALID_ARG;
+    if (r->n_rows >= (1ll << 31) - 256) return APE_ERR_LAYOUT;
+    return APE_OK;
+}
+
+bool span_ok(const ape_span_t& s, int64_t n_tokens) {
+    return s.len >= 0 && s.start >= 0 && s.start <= n_tokens && s.len <= n_tokens - s.start;
+}
+
+// bf16 [rows, heads, d] described to the copy engine as (d, heads, rows) with a 64-element (128-byte) swizzled box row.
+int make_map(ape_handle_t h, CUtensorMap* tm, const void* base, int d, int64_t heads, int64_t rows,
+             int64_t head_stride, int64_t token_stride, int box_heads, int box_rows) {
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(heads), static_cast<cuuint64_t>(rows)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(head_stride) * 2, static_cast<cuuint64_t>(token_stride) * 2};
+    cuuint32_t box[3] = {64u, static_cast<cuuint32_t>(box_heads), static_cast<cuuint32_t>(box_rows)};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    if (box_rows > 256 || box_heads > 256) return APE_ERR_LAYOUT;
+    const CUresult r = h->encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? APE_OK : APE_ERR_LAYOUT;
+}
+
+void add_span_tiles(std::vector<DevTile>& tiles, int64_t start, int64_t len, int tile, int32_t flags, int64_t grow_capacity) {
+    const int64_t extent = (flags & TILE_GROWS) ? grow_capacity : len;
+    for (int64_t off = 0; off < extent; off += tile) {
+        DevTile t;
+        t.tok = static_cast<int32_t>(start + off);
+        t.n_valid = static_cast<int32_t>(std::max<int64_t>(0, std::min<int64_t>(tile, len - off)));
+        t.key_base = static_cast<int32_t>(off);
+        t.flags = flags;
+        tiles.push_back(t);
+    }
+}
+
+// Context spans in any order -> sorted, with touching spans fused (Eq. 5 treats all contexts as one segment,
+// so boundaries between contexts do not matter to attend).
+std::vector<ape_span_t> fuse_spans(const ape_span_t* ctx, int n) {
+    std::vector<ape_span_t> v;
+    for (int i = 0; i < n; ++i) if (ctx[i].len > 0) v.push_back(ctx[i]);
+    std::sort(v.begin(), v.end(), [](const ape_span_t& a, const ape_span_t& b) { return a.start < b.start; });
+    std::vector<ape_span_t> out;
+    for (const auto& s : v) {
+        if (!out.empty() && out.back().start + out.back().len == s.start) out.back().len += s.len;
+        else out.push_back(s);
+    }
+    return out;
+}
+
+struct HostMeta {
+    std::vector<DevTile> tiles;
+    std::vector<DevItem> items;
+    std::vector<int32_t> cta_begin;
+    std::vector<DevReq> reqs;
+    std::vector<DevMerge> merge;
+};
+
+struct Run {   // a run of tiles of one segment for one (request, kv head, row-block group)
+    int req, kv_head, row_block, n_sib, seg, t0, t1, merge0;
+};
+
+// Split the concatenation of all runs evenly over n_bins bins (each bin = one CTA or one sibling group);
+// a run that straddles a bin boundary becomes several items, each with its own partial slot.
+void assign_stream(const std::vector<Run>& runs, int n_bins, int slot_mult, HostMeta& m) {
+    long long total = 0;
+    for (const auto& r : runs) total += r.t1 - r.t0;
+    const long long chunk = std::max<long long>(1, (total + n_bins - 1) / n_bins);
+    m.cta_begin.assign(1, 0);
+    long long room = chunk;
+    for (const auto& r : runs) {
+        int t = r.t0;
+        while (t < r.t1) {
+            const int take = static_cast<int>(std::min<long long>(room, r.t1 - t));
+            DevItem it;
+            it.req = r.req; it.kv_head = r.kv_head; it.row_block = r.row_block;
+            it.tile_begin = t; it.tile_end = t + take;
+            it.slot = static_cast<int32_t>(m.items.size()) * slot_mult;
+            it.seg = r.seg; it.n_sib = r.n_sib;
+            // bookkeeping for the merge: every live sibling's group record learns about this partial
+            for (int s = 0; s < r.n_sib; ++s) {
+                DevMerge& g = m.merge[r.merge0 + s];
+                g.slot_stride = slot_mult;
+                if (r.seg == SEG_CTX) { if (g.ctx_n == 0) g.ctx_slot0 = it.slot + s; g.ctx_n++; }
+                else { if (g.oth_n == 0) g.oth_slot0 = it.slot + s; g.oth_n++; }
+            }
+            m.items.push_back(it);
+            t += take; room -= take;
+            if (room == 0) { m.cta_begin.push_back(static_cast<int32_t>(m.items.size())); room = chunk; }
+        }
+    }
+    while (static_cast<int>(m.cta_begin.size()) < n_bins + 1) m.cta_begin.push_back(static_cast<int32_t>(m.items.size()));
+}
+
+int upload(ape_plan_t p, const HostMeta& m) {
+    auto rnd = [](size_t x) { return (x + 255) & ~size_t(255); };
+    const size_t b_tiles = rnd(m.tiles.size() * sizeof(DevTile) + 16), b_items = rnd(m.items.size() * sizeof(DevItem) + 16),
+                 b_cta = rnd(m.cta_begin.size() * 4 + 16), b_reqs = rnd(m.reqs.size() * sizeof(DevReq) + 16),
+                 b_merge = rnd(m.merge.size() * sizeof(DevMerge) + 16);
+    const size_t total = b_tiles + b_items + b_cta + b_reqs + b_merge;
+    std::vector<uint8_t> host(total, 0);
+    size_t o = 0;
+    auto put = [&](const void* src, size_t n, size_t padded) { if (n) std::memcpy(host.data() + o, src, n); size_t at = o; o += padded; return at; };
+    const size_t o_tiles = put(m.tiles.data(), m.tiles.size() * sizeof(DevTile), b_tiles);
+    const size_t o_items = put(m.items.data(), m.items.size() * sizeof(DevItem), b_items);
+    const size_t o_cta = put(m.cta_begin.data(), m.cta_begin.size() * 4, b_cta);
+    const size_t o_reqs = put(m.reqs.data(), m.reqs.size() * sizeof(DevReq), b_reqs);
+    const size_t o_merge = put(m.merge.data(), m.merge.size() * sizeof(DevMerge), b_merge);
+    if (cudaMalloc(&p->d_blob, total) != cudaSuccess) { p->d_blob = nullptr; return APE_ERR_NOMEM; }
+    if (cudaMemcpy(p->d_blob, host.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) return APE_ERR_CUDA;
+    uint8_t* b = static_cast<uint8_t*>(p->d_blob);
+    p->d_tiles = reinterpret_cast<DevTile*>(b + o_tiles);
+    p->d_items = reinterpret_cast<DevItem*>(b + o_items);
+    p->d_cta_begin = reinterpret_cast<int32_t*>(b + o_cta);
+    p->d_reqs = reinterpret_cast<DevReq*>(b + o_reqs);
+    p->d_merge = reinterpret_cast<DevMerge*>(b + o_merge);
+    p->n_items = static_cast<int>(m.items.size());
+    p->n_merge = static_cast<int>(m.merge.size());
+    return APE_OK;
+}
+
+RowsDesc rows_desc(const ape_rows_t& r) {
+    RowsDesc d; d.data = static_cast<__nv_bfloat16*>(r.data); d.token_stride = r.token_stride; d.head_stride = r.head_stride; return d;
+}
+
+int set_device(ape_handle_t h) { return cudaSetDevice(h->device) == cudaSuccess ? APE_OK : APE_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+int ape_create(ape_handle_t* handle, int device) {
+    if (!handle) return APE_ERR_INVALID_ARG;
+    *handle = nullptr;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess) return APE_ERR_CUDA;
+    if (device < 0 || device >= n_dev) return APE_ERR_INVALID_ARG;
+    ape_handle_t h = new (std::nothrow) ape_handle_s();
+    if (!h) return APE_ERR_NOMEM;
+    h->device = device;
+    cudaDeviceProp prop;
+    if (cudaSetDevice(device) != cudaSuccess || cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete h; return APE_ERR_CUDA; }
+    if (prop.major != 10) { delete h; return APE_ERR_CUDA; }      // the kernels are built for sm_100a only
+    h->n_sm = prop.multiProcessorCount;
+    h->smem_optin = prop.sharedMemPerBlockOptin;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) { delete h; return APE_ERR_CUDA; }
+    h->encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    if (cudaMalloc(&h->d_status, sizeof(int)) != cudaSuccess) { delete h; return APE_ERR_NOMEM; }
+    if (cudaMemset(h->d_status, 0, sizeof(int)) != cudaSuccess) { cudaFree(h->d_status); delete h; return APE_ERR_CUDA; }
+    *handle = h;
+    return APE_OK;
+}
+
+int ape_destroy(ape_handle_t h) {
+    if (!h) return APE_ERR_INVALID_ARG;
+    cudaSetDevice(h->device);
+    if (h->d_status) cudaFree(h->d_status);
+    delete h;
+    return APE_OK;
+}
+
+int ape_plan_destroy(ape_plan_t p) {
+    if (!p) return APE_ERR_INVALID_ARG;
+    if (p->d_blob) { cudaSetDevice(p->h->device); cudaFree(p->d_blob); }
+    delete p;
+    return APE_OK;
+}
+
+int ape_attend_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
+                    const ape_rows_t* out, float* lse, const ape_request_t* reqs, int32_t n_req, ape_mode_t mode,
+                    ape_plan_t* plan_out)
+{
+    if (!h || !plan_out) return APE_ERR_INVALID_ARG;
+    *plan_out = nullptr;
+    int G = 1; float c = 0.f;
+    int rc = check_shape(shape, &G, &c);              if (rc) return rc;
+    rc = check_pool(pool, shape);                     if (rc) return rc;
+    rc = check_rows(q, shape);                        if (rc) return rc;
+    rc = check_rows(out, shape);                      if (rc) return rc;
+    if (!reqs || n_req <= 0) return APE_ERR_INVALID_ARG;
+    if (mode != APE_PREFILL && mode != APE_DECODE) return APE_ERR_INVALID_ARG;
+    if (out->n_rows < q->n_rows) return APE_ERR_INVALID_ARG;
+    int64_t max_extra = INT64_MAX;
+    for (int r = 0; r < n_req; ++r) {
+        const ape_request_t& rq = reqs[r];
+        if (rq.q_len < 1 || rq.q_start < 0 || rq.q_start + rq.q_len > q->n_rows) return APE_ERR_INVALID_ARG;
+        if (mode == APE_DECODE && rq.q_len != 1) return APE_ERR_INVALID_ARG;
+        if (rq.n_ctx < 0 || (rq.n_ctx > 0 && !rq.ctx)) return APE_ERR_INVALID_ARG;
+        if (!span_ok(rq.prefix, pool->n_tokens) || !span_ok(rq.query_kv, pool->n_tokens)) return APE_ERR_INVALID_ARG;
+        for (int i = 0; i < rq.n_ctx; ++i) if (!span_ok(rq.ctx[i], pool->n_tokens)) return APE_ERR_INVALID_ARG;
+        if (rq.query_kv.len < rq.q_len) return APE_ERR_INVALID_ARG;
+        if (rq.query_kv_capacity < rq.query_kv.len || rq.query_kv.start + rq.query_kv_capacity > pool->n_tokens) return APE_ERR_INVALID_ARG;
+        max_extra = std::min(max_extra, rq.query_kv_capacity - rq.query_kv.len);
+    }
+    rc = set_device(h); if (rc) return rc;
+
+    ape_plan_t p = new (std::nothrow) ape_plan_s();
+    if (!p) return APE_ERR_NOMEM;
+    p->h = h; p->kind = (mode == APE_DECODE) ? PLAN_DECODE : PLAN_PREFILL;
+    p->shape = *shape; p->c = c; p->G = G; p->pool = *pool; p->q = *q; p->out = *out; p->lse = lse;
+    p->max_kv_extra = (mode == APE_DECODE) ? max_extra : 0;
+    const int D = shape->head_dim, H_kv = shape->n_kv_heads;
+
+    HostMeta m;
+    std::vector<Run> runs;
+    try {
+        if (mode == APE_DECODE) {
+            const int tile = kDecodeTile;
+            p->n_sib = 1;
+            m.merge.reserve(static_cast<size_t>(n_req) * H_kv);
+            for (int r = 0; r < n_req; ++r) {
+                const ape_request_t& rq = reqs[r];
+                DevReq dr{static_cast<int32_t>(rq.q_start), 1, static_cast<int32_t>(rq.query_kv.len), 0};
+                m.reqs.push_back(dr);
+                const int o0 = static_cast<int>(m.tiles.size());
+                add_span_tiles(m.tiles, rq.prefix.start, rq.prefix.len, tile, 0, 0);
+                add_span_tiles(m.tiles, rq.query_kv.start, rq.query_kv.len, tile, TILE_GROWS, rq.query_kv_capacity);
+                const int o1 = static_cast<int>(m.tiles.size());
+                for (const auto& s : fuse_spans(rq.ctx, rq.n_ctx)) add_span_tiles(m.tiles, s.start, s.len, tile, 0, 0);
+                const int c1 = static_cast<int>(m.tiles.size());
+                for (int hh = 0; hh < H_kv; ++hh) {
+                    DevMerge g{r, hh, 0, 0, 0, 0, 0, 1};
+                    const int mi = static_cast<int>(m.merge.size());
+                    m.merge.push_back(g);
+                    runs.push_back(Run{r, hh, 0, 1, SEG_OTHER, o0, o1, mi});
+                    if (c1 > o1) runs.push_back(Run{r, hh, 0, 1, SEG_CTX, o1, c1, mi});
+                }
+            }
+            p->n_cta = h->n_sm;
+            assign_stream(runs, p->n_cta, 1, m);
+            p->n_slots = static_cast<int>(m.items.size());
+            p->n_stages = decode_pick_stages(D, G, h->smem_optin - 2048);
+            if (p->n_stages < 2) { delete p; return APE_ERR_SHAPE; }
+            p->smem_bytes = decode_smem_bytes(D, G, p->n_stages);
+            const size_t rows = static_cast<size_t>(p->n_slots) * G;
+            p->ws_bytes = ((rows * D * 4 + 255) & ~size_t(255)) + ((rows * 2 * 4 + 255) & ~size_t(255));
+            rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
+            if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
+            if (!rc && decode_set_smem_attr(D, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+        } else {
+            const int tile = kAttnTileN;
+            const int TB = kAttnRows / G;                 // query tokens per row block
+            int max_rb = 1;
+            for (int r = 0; r < n_req; ++r) max_rb = std::max<int>(max_rb, static_cast<int>((reqs[r].q_len + TB - 1) / TB));
+            p->n_sib = std::min(4, max_rb);
+            const int n_groups = std::max(1, h->n_sm / p->n_sib);
+            for (int r = 0; r < n_req; ++r) {
+                const ape_request_t& rq = reqs[r];
+                DevReq dr{static_cast<int32_t>(rq.q_start), static_cast<int32_t>(rq.q_len), static_cast<int32_t>(rq.query_kv.len), 0};
+                m.reqs.push_back(dr);
+                const int o0 = static_cast<int>(m.tiles.size());
+                add_span_tiles(m.tiles, rq.prefix.start, rq.prefix.len, tile, 0, 0);
+                add_span_tiles(m.tiles, rq.query_kv.start, rq.query_kv.len, tile, TILE_CAUSAL, 0);
+                const int o1 = static_cast<int>(m.tiles.size());
+                for (const auto& s : fuse_spans(rq.ctx, rq.n_ctx)) add_span_tiles(m.tiles, s.start, s.len, tile, 0, 0);
+                const int c1 = static_cast<int>(m.tiles.size());
+                const int RB = static_cast<int>((rq.q_len + TB - 1) / TB);
+                for (int hh = 0; hh < H_kv; ++hh) {
+                    for (int rb0 = 0; rb0 < RB; rb0 += p->n_sib) {
+                        const int live = std::min(p->n_sib, RB - rb0);
+                        const int mi = static_cast<int>(m.merge.size());
+                        for (int s = 0; s < live; ++s) m.merge.push_back(DevMerge{r, hh, rb0 + s, 0, 0, 0, 0, 1});
+                        runs.push_back(Run{r, hh, rb0, live, SEG_OTHER, o0, o1, mi});
+                        if (c1 > o1) runs.push_back(Run{r, hh, rb0, live, SEG_CTX, o1, c1, mi});
+                    }
+                }
+            }
+            assign_stream(runs, n_groups, p->n_sib, m);
+            p->n_cta = n_groups * p->n_sib;
+            p->n_slots = static_cast<int>(m.items.size()) * p->n_sib;
+            p->smem_bytes = attn_smem_bytes(D);
+            const size_t rows = static_cast<size_t>(p->n_slots) * kAttnRows;
+            p->ws_bytes = ((rows * D * 4 + 255) & ~size_t(255)) + ((rows * 2 * 4 + 255) & ~size_t(255));
+            rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
+            if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
+            if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
+            if (!rc && attn_set_smem_attr(D, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+        }
+        if (!rc) rc = upload(p, m);
+    } catch (const std::bad_alloc&) {
+        rc = APE_ERR_NOMEM;
+    }
+    if (rc) { ape_plan_destroy(p); return rc; }
+    *plan_out = p;
+    return APE_OK;
+}
+
+int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
+                    const ape_rows_t* out, float* lse, const ape_span_t* prefix, const ape_span_t* ctx, int32_t n_ctx,
+                    ape_plan_t* plan_out)
+{
+    if (!h || !plan_out) return APE_ERR_INVALID_ARG;
+    *plan_out = nullptr;
+    int G = 1; float c = 0.f;
+    int rc = check_shape(shape, &G, &c);              if (rc) return rc;
+    rc = check_pool(pool, shape);                     if (rc) return rc;
+    rc = check_rows(q, shape);                        if (rc) return rc;
+    rc = check_rows(out, shape);                      if (rc) return rc;
+    if (!prefix || n_ctx < 0 || (n_ctx > 0 && !ctx)) return APE_ERR_INVALID_ARG;
+    if (!span_ok(*prefix, pool->n_tokens)) return APE_ERR_INVALID_ARG;
+    for (int i = 0; i < n_ctx; ++i) {
+        if (!span_ok(ctx[i], pool->n_tokens)) return APE_ERR_INVALID_ARG;
+        if (ctx[i].start + ctx[i].len > q->n_rows || ctx[i].start + ctx[i].len > out->n_rows) return APE_ERR_INVALID_ARG;
+    }
+    rc = set_device(h); if (rc) return rc;
+
+    ape_plan_t p = new (std::nothrow) ape_plan_s();
+    if (!p) return APE_ERR_NOMEM;
+    p->h = h; p->kind = PLAN_ENCODE; p->shape = *shape; p->c = c; p->G = G; p->pool = *pool; p->q = *q; p->out = *out; p->lse = lse;
+    p->n_sib = 1;
+    const int D = shape->head_dim, H_kv = shape->n_kv_heads, tile = kAttnTileN, TB = kAttnRows / G;
+
+    HostMeta m;
+    try {
+        struct Work { DevItem it; long long cost; };
+        std::vector<Work> work;
+        for (int i = 0; i < n_ctx; ++i) {
+            DevReq dr{static_cast<int32_t>(ctx[i].start), static_cast<int32_t>(ctx[i].len), static_cast<int32_t>(ctx[i].len), 0};
+            m.reqs.push_back(dr);
+            if (ctx[i].len == 0) continue;
+            const int t0 = static_cast<int>(m.tiles.size());
+            add_span_tiles(m.tiles, prefix->start, prefix->len, tile, 0, 0);
+            const int n_pref = static_cast<int>(m.tiles.size()) - t0;
+            add_span_tiles(m.tiles, ctx[i].start, ctx[i].len, tile, TILE_CAUSAL, 0);
+            const int t1 = static_cast<int>(m.tiles.size());
+            const int RB = static_cast<int>((ctx[i].len + TB - 1) / TB);
+            for (int hh = 0; hh < H_kv; ++hh)
+                for (int rb = 0; rb < RB; ++rb) {
+                    const int64_t last_tok = std::min<int64_t>(ctx[i].len, static_cast<int64_t>(rb + 1) * TB) - 1;
+                    const int vis = n_pref + static_cast<int>(last_tok / tile) + 1;     // tiles this row block can see
+                    DevItem it{i, hh, rb, t0, std::min(t1, t0 + vis), 0, SEG_FINAL, 1};
+                    work.push_back(Work{it, vis});
+                }
+        }
+        // longest-first round robin over the CTAs keeps the per-CTA tile counts close
+        std::stable_sort(work.begin(), work.end(), [](const Work& a, const Work& b) { return a.cost > b.cost; });
+        p->n_cta = std::max(1, std::min<int>(h->n_sm, static_cast<int>(work.size())));
+        std::vector<std::vector<DevItem>> bins(p->n_cta);
+        std::vector<long long> load(p->n_cta, 0);
+        for (size_t w = 0; w < work.size(); ++w) {
+            int b = static_cast<int>(std::min_element(load.begin(), load.end()) - load.begin());
+            bins[b].push_back(work[w].it); load[b] += work[w].cost;
+        }
+        m.cta_begin.push_back(0);
+        for (auto& b : bins) { for (auto& it : b) m.items.push_back(it); m.cta_begin.push_back(static_cast<int32_t>(m.items.size())); }
+        p->n_slots = 0;
+        p->ws_bytes = 0;
+        p->smem_bytes = attn_smem_bytes(D);
+        rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
+        if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
+        if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
+        if (!rc && attn_set_smem_attr(D, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+        if (!rc) rc = upload(p, m);
+    } catch (const std::bad_alloc&) {
+        rc = APE_ERR_NOMEM;
+    }
+    if (rc) { ape_plan_destroy(p); return rc; }
+    *plan_out = p;
+    return APE_OK;
+}
+
+int ape_plan_workspace_bytes(ape_plan_t p, size_t* bytes) {
+    if (!p || !bytes) return APE_ERR_INVALID_ARG;
+    *bytes = p->ws_bytes;
+    return APE_OK;
+}
+
+int ape_plan_last_launches(ape_plan_t p, int32_t* n) {
+    if (!p || !n) return APE_ERR_INVALID_ARG;
+    *n = p->last_launches;
+    return APE_OK;
+}
+
+int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace, size_t ws_bytes, void* stream_v) {
+    if (!p) return APE_ERR_INVALID_ARG;
+    if (p->kind != PLAN_PREFILL && p->kind != PLAN_DECODE) return APE_ERR_MODE;
+    if (!(T > 0.f) || !(S > 0.f) || !std::isfinite(T) || !std::isfinite(S)) return APE_ERR_RANGE;
+    if (kv_extra < 0 || kv_extra > p->max_kv_extra) return APE_ERR_RANGE;
+    if (p->ws_bytes > 0 && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || ws_bytes < p->ws_bytes)) return APE_ERR_WORKSPACE;
+    int rc = set_device(p->h); if (rc) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const int D = p->shape.head_dim, G = p->G;
+    constexpr float kLog2e = 1.4426950408889634f;
+    const int rows_per_slot = (p->kind == PLAN_DECODE) ? G : kAttnRows;
+    const size_t rows = static_cast<size_t>(p->n_slots) * rows_per_slot;
+    float* ws_o = static_cast<float*>(workspace);
+    float* ws_ml = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + ((rows * D * 4 + 255) & ~size_t(255)));
+    p->last_launches = 0;
+
+    if (p->kind == PLAN_DECODE) {
+        DecodeParams dp;
+        dp.tiles = p->d_tiles; dp.items = p->d_items; dp.cta_item_begin = p->d_cta_begin; dp.reqs = p->d_reqs;
+        dp.q = rows_desc(p->q); dp.ws_o = ws_o; dp.ws_ml = ws_ml;
+        dp.scale_oth_log2 = p->c * kLog2e; dp.scale_ctx_log2 = p->c / T * kLog2e;
+        dp.kv_extra = static_cast<int32_t>(kv_extra); dp.G = G; dp.n_stages = p->n_stages; dp.status = p->h->d_status;
+        if (launch_decode(D, p->tm_k, p->tm_v, dp, p->n_cta, p->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
+    } else {
+        AttnParams ap;
+        ap.tiles = p->d_tiles; ap.items = p->d_items; ap.cta_item_begin = p->d_cta_begin; ap.reqs = p->d_reqs;
+        ap.out = rows_desc(p->out); ap.lse_out = nullptr; ap.ws_o = ws_o; ap.ws_ml = ws_ml;
+        ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c / T * kLog2e;
+        ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = p->n_sib; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
+        if (launch_attn(D, p->tm_q, p->tm_k, p->tm_v, ap, p->n_cta, p->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
+    }
+    p->last_launches++;
+
+    MergeParams mp;
+    mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.n_groups = p->n_merge; mp.rows_per_slot = rows_per_slot;
+    mp.tokens_per_block = rows_per_slot / G; mp.ws_o = ws_o; mp.ws_ml = ws_ml; mp.out = rows_desc(p->out); mp.lse_out = p->lse;
+    mp.S = S; mp.G = G; mp.H_q = p->shape.n_q_heads; mp.D = D;
+    if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;
+    p->last_launches++;
+    return APE_OK;
+}
+
+int ape_encode_contexts(ape_plan_t p, void* workspace, size_t ws_bytes, void* stream_v) {
+    (void)workspace; (void)ws_bytes;
+    if (!p) return APE_ERR_INVALID_ARG;
+    if (p->kind != PLAN_ENCODE) return APE_ERR_MODE;
+    int rc = set_device(p->h); if (rc) return rc;
+    p->last_launches = 0;
+    if (p->n_items == 0) return APE_OK;
+    constexpr float kLog2e = 1.4426950408889634f;
+    AttnParams ap;
+    ap.tiles = p->d_tiles; ap.items = p->d_items; ap.cta_item_begin = p->d_cta_begin; ap.reqs = p->d_reqs;
+    ap.out = rows_desc(p->out); ap.lse_out = p->lse; ap.ws_o = nullptr; ap.ws_ml = nullptr;
+    ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c * kLog2e;
+    ap.G = p->G; ap.H_q = p->shape.n_q_heads; ap.n_sib = 1; ap.q_rows_are_pool = 1; ap.status = p->h->d_status;
+    if (launch_attn(p->shape.head_dim, p->tm_q, p->tm_k, p->tm_v, ap, p->n_cta, p->smem_bytes,
+                    static_cast<cudaStream_t>(stream_v)) != cudaSuccess) return APE_ERR_CUDA;
+    p->last_launches = 1;
+    return APE_OK;
+}
+
+int ape_attend_host(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace, size_t ws_bytes,
+                    const void* h_q, const void* h_k, const void* h_v, void* h_out,
+                    size_t* h2d_bytes, size_t* d2h_bytes, void* stream_v) {
+    if (!p || !h_q || !h_k || !h_v || !h_out) return APE_ERR_INVALID_ARG;
+    if (p->kind != PLAN_PREFILL && p->kind != PLAN_DECODE) return APE_ERR_MODE;
+    int rc = set_device(p->h); if (rc) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const size_t qb = static_cast<size_t>(p->q.n_rows) * p->q.token_stride * 2;
+    const size_t kb = static_cast<size_t>(p->pool.n_tokens) * p->pool.token_stride * 2;
+    const size_t ob = static_cast<size_t>(p->q.n_rows) * p->out.token_stride * 2;
+    if (cudaMemcpyAsync(p->q.data, h_q, qb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return APE_ERR_CUDA;
+    if (cudaMemcpyAsync(const_cast<void*>(p->pool.k), h_k, kb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return APE_ERR_CUDA;
+    if (cudaMemcpyAsync(const_cast<void*>(p->pool.v), h_v, kb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return APE_ERR_CUDA;
+    rc = ape_attend(p, T, S, kv_extra, workspace, ws_bytes, stream_v);
+    if (rc) return rc;
+    if (cudaMemcpyAsync(h_out, p->out.data, ob, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return APE_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return APE_ERR_CUDA;
+    if (h2d_bytes) *h2d_bytes = qb + 2 * kb;
+    if (d2h_bytes) *d2h_bytes = ob;
+    return APE_OK;
+}
+
+int ape_get_status(ape_handle_t h, int32_t* device_status) {
+    if (!h || !device_status) return APE_ERR_INVALID_ARG;
+    int rc = set_device(h); if (rc) return rc;
+    if (cudaDeviceSynchronize() != cudaSuccess) return APE_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpy(&v, h->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return APE_ERR_CUDA;
+    if (v != 0 && cudaMemset(h->d_status, 0, sizeof(int)) != cudaSuccess) return APE_ERR_CUDA;
+    *device_status = v;
+    return APE_OK;
+}
+
+const char* ape_status_string(int s) {
+    switch (s) {
+        case APE_OK: return "ok";
+        case APE_ERR_INVALID_ARG: return "invalid argument";
+        case APE_ERR_SHAPE: return "unsupported head shape";
+        case APE_ERR_ALIGN: return "pointer or stride not aligned";
+        case APE_ERR_RANGE: return "value out of range";
+        case APE_ERR_LAYOUT: return "tensor layout cannot be described to the copy engine";
+        case APE_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case APE_ERR_CUDA: return "CUDA call failed";
+        case APE_ERR_TIMEOUT: return "a kernel gave up on a bounded wait";
+        case APE_ERR_NOMEM: return "out of memory";
+        case APE_ERR_MODE: return "plan used with the wrong entry point";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"
