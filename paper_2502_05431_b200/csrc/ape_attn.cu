@@ -1,0 +1,462 @@
+// Tensor-core attention kernel of libape, shared by query prefill (ape_attend) and context encoding
+// (ape_encode_contexts).  One persistent CTA owns a block of 256 packed query rows (row = token * G + head-in-group,
+// so the G query heads of a KV head share every K/V tile) as two 128-row halves, and walks its list of work items.
+// Every item is a run of 128-key tiles of ONE segment, so a plain online softmax per item is exact; the scaling
+// factor S of Eq. 5 acts on whole-segment log-sum-exps and is applied by the merge kernel afterwards.
+//
+// Roles (warp-specialised, 320 threads):
+//   warps 0-3 / 4-7  softmax of half 0 / half 1: one thread per row; S is read from TMEM, P = 2^(s - m) goes back
+//                    to TMEM as bf16 over the S columns, the running sum stays in a register; also the epilogue
+//   warp 8           producer: bulk tensor copies of Q, K and V tiles into 128-byte-swizzled shared memory
+//   warp 9           MMA issuer: S = Q K^T (both operands in shared memory) and O += P V (P from TMEM) with
+//                    tcgen05.mma, accumulators in TMEM; owns the TMEM allocation
+// The two halves run one tile apart, so that the tensor pipe works on one half while the other does its exponentials.
+#include "ape_common.cuh"
+#include "ape_kernels.h"
+#include "ape_tcgen05.cuh"
+
+namespace ape {
+
+namespace {
+
+constexpr int kTileN = kAttnTileN;            // 128 keys per tile
+constexpr int kHalfRows = 128;
+constexpr int kThreads = 320;
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp = 9;
+constexpr int kNK = 2;                        // K stages
+constexpr int kNV = 2;                        // V stages
+constexpr int kSlabBytes = 128 * 128;         // 128 rows x 64 bf16
+constexpr float kRescaleThreshold = 8.0f;     // base-2 units: O is rescaled only when the row maximum grew by more
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct ItemGeom {
+    int rb;          // row block of this CTA for the item
+    int last_tok;    // last live query token of the row block
+    int off;         // l_k - q_len: causal offset
+};
+
+__device__ __forceinline__ bool tile_visible(const DevTile& t, const ItemGeom& g) {
+    if (t.n_valid <= 0) return false;
+    if ((t.flags & TILE_CAUSAL) && t.key_base > g.last_tok + g.off) return false;
+    return true;
+}
+
+}  // namespace
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const AttnParams p)
+{
+    constexpr int kSlabs = D / 64;
+    constexpr int kTileBytes = kSlabs * kSlabBytes;            // one K or V tile, also one Q half
+    constexpr uint32_t kTmemCols = 512;
+    constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 256 + D;
+    constexpr uint32_t kIdescQK = idesc_bf16_f32(128, kTileN, 0, 0);
+    constexpr uint32_t kIdescPV = idesc_bf16_f32(128, D, 0, 1);
+
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* q_smem = smem;                                    // 2 halves
+    uint8_t* k_smem = q_smem + 2 * kTileBytes;                 // kNK stages
+    uint8_t* v_smem = k_smem + kNK * kTileBytes;               // kNV stages
+    uint64_t* bars = reinterpret_cast<uint64_t*>(v_smem + kNV * kTileBytes);
+    // barrier map
+    const uint32_t bar0 = smem_u32(bars);
+    const uint32_t bar_q_full = bar0, bar_q_empty = bar0 + 8;
+    const uint32_t bar_k_full = bar0 + 16, bar_k_empty = bar_k_full + 8 * kNK;
+    const uint32_t bar_v_full = bar_k_empty + 8 * kNK, bar_v_empty = bar_v_full + 8 * kNV;
+    const uint32_t bar_s_full = bar_v_empty + 8 * kNV;         // [2]
+    const uint32_t bar_p_full = bar_s_full + 16;               // [2]
+    const uint32_t bar_o_full = bar_p_full + 16;               // [2]
+    const uint32_t bar_done = bar_o_full + 16;
+    __shared__ uint32_t tmem_base_smem;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(bar_q_full, 1); mbar_init(bar_q_empty, 1);
+        for (int s = 0; s < kNK; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 1); }
+        for (int s = 0; s < kNV; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 1); }
+        for (int w = 0; w < 2; ++w) {
+            mbar_init(bar_s_full + 8 * w, 1);
+            mbar_init(bar_p_full + 8 * w, kHalfRows);
+            mbar_init(bar_o_full + 8 * w, 1);
+        }
+        mbar_init(bar_done, 1);
+        mbar_fence_init();
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(smem_u32(&tmem_base_smem), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_smem;
+
+    const int n_sib = p.n_sib;
+    const int group = blockIdx.x / n_sib, sib = blockIdx.x - group * n_sib;
+    const int item_begin = p.cta_item_begin[group], item_end = p.cta_item_begin[group + 1];
+    const int G = p.G;
+    const int TB = kAttnRows / G;            // query tokens per row block
+
+    auto geom = [&](const DevItem& item, const DevReq& rq) {
+        ItemGeom g;
+        g.rb = item.row_block + sib;
+        g.last_tok = min(rq.q_len, (g.rb + 1) * TB) - 1;
+        g.off = rq.l_k - rq.q_len;
+        return g;
+    };
+
+    if (warp == kProducerWarp) {
+        // =============================== producer ====================================================================
+        if (lane == 0) {
+            tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
+            uint32_t kcnt = 0, vcnt = 0, q_loads = 0;
+            int last_req = -1, last_head = -1, last_rb = -1;
+            bool ok = true;
+            for (int it = item_begin; it < item_end && ok; ++it) {
+                const DevItem item = p.items[it];
+                if (sib >= item.n_sib) continue;
+                const DevReq rq = p.reqs[item.req];
+                const ItemGeom g = geom(item, rq);
+                if (!(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
+                    if (q_loads > 0 && !mbar_wait(bar_q_empty, (q_loads - 1) & 1, &abort_flag, p.status)) { ok = false; break; }
+                    mbar_expect_tx(bar_q_full, 2 * kTileBytes);
+                    #pragma unroll
+                    for (int w = 0; w < 2; ++w) {
+                        const int tok0 = rq.q_row0 + g.rb * TB + w * (kHalfRows / G);
+                        #pragma unroll
+                        for (int sl = 0; sl < kSlabs; ++sl)
+                            tma_load_3d(smem_u32(q_smem + w * kTileBytes + sl * kSlabBytes), &tm_q, bar_q_full,
+                                        sl * 64, item.kv_head * G, tok0);
+                    }
+                    ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
+                }
+                for (int t = item.tile_begin; t < item.tile_end; ++t) {
+                    const DevTile tile = p.tiles[t];
+                    if (!tile_visible(tile, g)) continue;
+                    {
+                        const int s = kcnt % kNK; const uint32_t use = kcnt / kNK;
+                        if (!mbar_wait(bar_k_empty + 8 * s, (use & 1) ^ 1, &abort_flag, p.status)) { ok = false; break; }
+                        mbar_expect_tx(bar_k_full + 8 * s, kTileBytes);
+                        #pragma unroll
+                        for (int sl = 0; sl < kSlabs; ++sl)
+                            tma_load_3d(smem_u32(k_smem + s * kTileBytes + sl * kSlabBytes), &tm_k, bar_k_full + 8 * s,
+                                        sl * 64, item.kv_head, tile.tok);
+                        ++kcnt;
+                    }
+                    {
+                        const int s = vcnt % kNV; const uint32_t use = vcnt / kNV;
+                        if (!mbar_wait(bar_v_empty + 8 * s, (use & 1) ^ 1, &abort_flag, p.status)) { ok = false; break; }
+                        mbar_expect_tx(bar_v_full + 8 * s, kTileBytes);
+                        #pragma unroll
+                        for (int sl = 0; sl < kSlabs; ++sl)
+                            tma_load_3d(smem_u32(v_smem + s * kTileBytes + sl * kSlabBytes), &tm_v, bar_v_full + 8 * s,
+                                        sl * 64, item.kv_head, tile.tok);
+                        ++vcnt;
+                    }
+                }
+            }
+            if (!ok) {
+                // wait (bounded) for copies that were issued but whose barrier nobody may consume any more
+                const long long t0 = clock64();
+                for (int s = 0; s < kNK; ++s) {
+                    const uint32_t issued = (kcnt > static_cast<uint32_t>(s)) ? (kcnt - 1 - s) / kNK + 1 : 0;
+                    while (issued && !mbar_try_wait(bar_k_full + 8 * s, (issued - 1) & 1) && clock64() - t0 < (1ll << 24)) {}
+                }
+                for (int s = 0; s < kNV; ++s) {
+                    const uint32_t issued = (vcnt > static_cast<uint32_t>(s)) ? (vcnt - 1 - s) / kNV + 1 : 0;
+                    while (issued && !mbar_try_wait(bar_v_full + 8 * s, (issued - 1) & 1) && clock64() - t0 < (1ll << 24)) {}
+                }
+                while (q_loads && !mbar_try_wait(bar_q_full, (q_loads - 1) & 1) && clock64() - t0 < (1ll << 24)) {}
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // =============================== MMA issuer ==================================================================
+        // All 32 lanes walk the loop and take part in the waits; lane 0 issues the tensor-core instructions.
+        uint32_t kcnt = 0, vcnt = 0, q_loads = 0, pcnt = 0;
+        int last_req = -1, last_head = -1, last_rb = -1;
+        bool ok = true;
+        const uint32_t tS[2] = {tmem_base + kColS0, tmem_base + kColS1};
+        const uint32_t tO[2] = {tmem_base + kColO0, tmem_base + kColO1};
+        auto wait_all = [&](uint32_t bar, uint32_t parity) {
+            return __all_sync(0xffffffffu, mbar_wait(bar, parity, &abort_flag, p.status)) != 0;
+        };
+        auto issue_qk = [&](int w, uint32_t k_base) {
+            const uint32_t q_base = smem_u32(q_smem + w * kTileBytes);
+            #pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+                const uint32_t o = (ks >> 2) * kSlabBytes + (ks & 3) * 32;
+                mma_ss(tS[w], smem_desc_sw128(q_base + o, 16, 1024), smem_desc_sw128(k_base + o, 16, 1024), kIdescQK, ks > 0);
+            }
+        };
+        auto issue_pv = [&](int w, uint32_t v_base, bool accumulate) {
+            #pragma unroll
+            for (int ks = 0; ks < kTileN / 16; ++ks)
+                mma_ts(tO[w], tS[w] + ks * 8, smem_desc_sw128(v_base + ks * 2048, kSlabBytes, 1024), kIdescPV,
+                       (accumulate || ks > 0) ? 1u : 0u);
+        };
+        // V rows past the span may hold anything (even NaN bit patterns); P is 0 there, and 0 * NaN must stay 0.
+        auto scrub_v = [&](uint8_t* v_tile, int n_valid) {
+            const int per_slab = (kTileN - n_valid) * 8;              // 16-byte chunks to clear in each slab
+            for (int i = lane; i < per_slab * kSlabs; i += 32) {
+                const int sl = i / per_slab, rem = i - sl * per_slab;
+                *reinterpret_cast<uint4*>(v_tile + sl * kSlabBytes + (n_valid + (rem >> 3)) * 128 + (rem & 7) * 16) = make_uint4(0, 0, 0, 0);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+        };
+
+        for (int it = item_begin; it < item_end && ok; ++it) {
+            const DevItem item = p.items[it];
+            if (sib >= item.n_sib) continue;
+            const DevReq rq = p.reqs[item.req];
+            const ItemGeom g = geom(item, rq);
+            if (!(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
+                if (q_loads > 0 && lane == 0) mma_commit(bar_q_empty);     // Q may be replaced once every MMA so far is done
+                if (!wait_all(bar_q_full, q_loads & 1)) { ok = false; break; }
+                ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
+            }
+            bool have_prev = false, o_started = false;
+            int prev_valid = kTileN;
+            uint32_t prev_vs = 0, prev_vphase = 0;
+            for (int t = item.tile_begin; t < item.tile_end; ++t) {
+                const DevTile tile = p.tiles[t];
+                if (!tile_visible(tile, g)) continue;
+                const int ksn = kcnt % kNK;
+                if (!wait_all(bar_k_full + 8 * ksn, (kcnt / kNK) & 1)) { ok = false; break; }
+                const uint32_t k_base = smem_u32(k_smem + ksn * kTileBytes);
+                ++kcnt;
+                const uint32_t vs = vcnt % kNV, vphase = (vcnt / kNV) & 1;
+                ++vcnt;
+                if (!have_prev) {
+                    tc_fence_after();
+                    if (lane == 0) {
+                        issue_qk(0, k_base); mma_commit(bar_s_full);
+                        issue_qk(1, k_base); mma_commit(bar_s_full + 8);
+                        mma_commit(bar_k_empty + 8 * ksn);
+                    }
+                    __syncwarp();
+                } else {
+                    // previous tile: O += P V, interleaved half by half with this tile's S = Q K^T
+                    if (!wait_all(bar_v_full + 8 * prev_vs, prev_vphase)) { ok = false; break; }
+                    uint8_t* v_tile = v_smem + prev_vs * kTileBytes;
+                    if (prev_valid < kTileN) scrub_v(v_tile, prev_valid);
+                    const uint32_t v_base = smem_u32(v_tile);
+                    for (int w = 0; w < 2; ++w) {
+                        if (!wait_all(bar_p_full + 8 * w, pcnt & 1)) { ok = false; break; }
+                        tc_fence_after();
+                        if (lane == 0) {
+                            issue_pv(w, v_base, o_started);
+                            if (w == 1) mma_commit(bar_v_empty + 8 * prev_vs);
+                            issue_qk(w, k_base); mma_commit(bar_s_full + 8 * w);
+                            if (w == 1) mma_commit(bar_k_empty + 8 * ksn);
+                        }
+                        __syncwarp();
+                    }
+                    if (!ok) break;
+                    ++pcnt; o_started = true;
+                }
+                have_prev = true; prev_valid = tile.n_valid; prev_vs = vs; prev_vphase = vphase;
+            }
+            if (ok && have_prev) {
+                // drain: the last tile's O += P V; o_full tells the softmax threads that O is final
+                if (!wait_all(bar_v_full + 8 * prev_vs, prev_vphase)) { ok = false; break; }
+                uint8_t* v_tile = v_smem + prev_vs * kTileBytes;
+                if (prev_valid < kTileN) scrub_v(v_tile, prev_valid);
+                const uint32_t v_base = smem_u32(v_tile);
+                for (int w = 0; w < 2; ++w) {
+                    if (!wait_all(bar_p_full + 8 * w, pcnt & 1)) { ok = false; break; }
+                    tc_fence_after();
+                    if (lane == 0) {
+                        issue_pv(w, v_base, o_started);
+                        mma_commit(bar_o_full + 8 * w);
+                        if (w == 1) mma_commit(bar_v_empty + 8 * prev_vs);
+                    }
+                    __syncwarp();
+                }
+                ++pcnt;
+            }
+        }
+        if (!ok) {
+            // let the tensor pipe drain (bounded) before the tensor memory is released
+            if (lane == 0) mma_commit(bar_done);
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar_done, 0) && clock64() - t0 < (1ll << 24)) {}
+        }
+    } else {
+        // =============================== softmax + epilogue ==========================================================
+        const int w = warp >> 2;
+        const int r_local = (warp & 3) * 32 + lane;
+        const int R = w * kHalfRows + r_local;                      // row inside the 256-row block
+        const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + lane_base + (w ? kColS1 : kColS0);
+        const uint32_t tO = tmem_base + lane_base + (w ? kColO1 : kColO0);
+        const uint32_t my_s_full = bar_s_full + 8 * w, my_p_full = bar_p_full + 8 * w, my_o_full = bar_o_full + 8 * w;
+        uint32_t scnt = 0, ocnt = 0;
+        bool ok = true;
+
+        for (int it = item_begin; it < item_end && ok; ++it) {
+            const DevItem item = p.items[it];
+            if (sib >= item.n_sib) continue;
+            const DevReq rq = p.reqs[item.req];
+            const ItemGeom g = geom(item, rq);
+            const int tok = g.rb * TB + R / G;
+            const int hg = R % G;
+            const bool live = tok < rq.q_len;
+            const float scale = (item.seg == SEG_CTX) ? p.scale_ctx_log2 : p.scale_oth_log2;
+            float m = -INFINITY, l = 0.f;
+            int n_local = 0;
+
+            for (int t = item.tile_begin; t < item.tile_end; ++t) {
+                const DevTile tile = p.tiles[t];
+                if (!tile_visible(tile, g)) continue;
+                if (!__all_sync(0xffffffffu, mbar_wait(my_s_full, scnt & 1, &abort_flag, p.status))) { ok = false; break; }
+                ++scnt;
+                tc_fence_after();
+                float s[kTileN];
+                {
+                    uint32_t (*sr)[32] = reinterpret_cast<uint32_t (*)[32]>(s);
+                    #pragma unroll
+                    for (int c = 0; c < kTileN / 32; ++c) tmem_ld32(tS + c * 32, sr[c]);
+                    tmem_ld_wait();
+                }
+                int limit = tile.n_valid;
+                if (tile.flags & TILE_CAUSAL) limit = min(limit, tok + g.off - tile.key_base + 1);
+                if (limit < kTileN) {
+                    #pragma unroll
+                    for (int i = 0; i < kTileN; ++i) s[i] = (i < limit) ? s[i] : -INFINITY;
+                }
+                float mx = s[0];
+                #pragma unroll
+                for (int i = 1; i < kTileN; ++i) mx = fmaxf(mx, s[i]);
+                const float m_new = fmaxf(m, mx * scale);
+                if (n_local == 0) {
+                    m = m_new;
+                } else {
+                    const bool grow = m_new > m + kRescaleThreshold;
+                    if (__any_sync(0xffffffffu, grow)) {
+                        // S of this tile is complete, so every earlier O += P V of this half is complete too, and the
+                        // next one cannot start before this thread has published P: O is quiescent here.
+                        const float f = grow ? fast_exp2(m - m_new) : 1.f;
+                        l *= f;
+                        #pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c * 32, o);
+                            tmem_ld_wait();
+                            #pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                            tmem_st32(tO + c * 32, o);
+                        }
+                        tmem_st_wait();
+                        if (grow) m = m_new;
+                    }
+                }
+                const float m_use = (m == -INFINITY) ? 0.f : m;
+                float sum = 0.f;
+                #pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    uint32_t pk[32];
+                    #pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float p0 = fast_exp2(fmaf(s[hh * 64 + 2 * i], scale, -m_use));
+                        const float p1 = fast_exp2(fmaf(s[hh * 64 + 2 * i + 1], scale, -m_use));
+                        sum += p0 + p1;
+                        pk[i] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st32(tS + hh * 32, pk);
+                }
+                l += sum;
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(my_p_full);
+                ++n_local;
+            }
+            if (!ok) break;
+
+            // ---- epilogue of the item -------------------------------------------------------------------------------
+            if (n_local > 0) {
+                if (!__all_sync(0xffffffffu, mbar_wait(my_o_full, ocnt & 1, &abort_flag, p.status))) { ok = false; break; }
+                ++ocnt;
+                tc_fence_after();
+            }
+            if (item.seg == SEG_FINAL) {
+                const float inv = (l > 0.f) ? 1.f / l : 0.f;
+                const int h = item.kv_head * G + hg;
+                __nv_bfloat16* dst = p.out.data + static_cast<int64_t>(rq.q_row0 + tok) * p.out.token_stride
+                                     + static_cast<int64_t>(h) * p.out.head_stride;
+                #pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
+                    tmem_ld_wait();
+                    if (live) {
+                        #pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint4 v;
+                            v.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
+                            v.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
+                            v.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
+                            v.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
+                            *reinterpret_cast<uint4*>(dst + c * 32 + i * 8) = v;
+                        }
+                    }
+                }
+                if (live && p.lse_out != nullptr)
+                    p.lse_out[static_cast<int64_t>(rq.q_row0 + tok) * p.H_q + h] = (l > 0.f) ? (m + fast_log2(l)) * kLn2 : -INFINITY;
+            } else {
+                const size_t row = static_cast<size_t>(item.slot + sib) * kAttnRows + R;
+                if (n_local > 0) {
+                    float* dst = p.ws_o + row * D;
+                    #pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c * 32, o);
+                        tmem_ld_wait();
+                        if (live) {
+                            #pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                *reinterpret_cast<uint4*>(dst + c * 32 + i * 4) = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+                        }
+                    }
+                }
+                if (live) *reinterpret_cast<float2*>(p.ws_ml + row * 2) = make_float2(m, (n_local > 0) ? l : 0.f);
+            }
+        }
+    }
+
+    // ---- teardown: every role has left its loop (normally or on an abort) ----------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+size_t attn_smem_bytes(int D) {
+    const size_t tile = static_cast<size_t>(D / 64) * kSlabBytes;
+    return 1024 + (2 + kNK + kNV) * tile + 256;
+}
+
+cudaError_t attn_set_smem_attr(int D, size_t smem_bytes) {
+    if (D == 128)
+        return cudaFuncSetAttribute(ape_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes));
+    return cudaFuncSetAttribute(ape_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes));
+}
+
+cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                        const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream)
+{
+    if (D == 128) ape_attn_kernel<128><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
+    else ape_attn_kernel<64><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
+    return cudaGetLastError();
+}
+
+}  // namespace ape
