@@ -1,0 +1,219 @@
+"""Thin ctypes binding over libape.so (C ABI: include/ape.h).  Argument marshalling only.
+
+Every step of the attention path runs in the library's CUDA kernels; there is no Python or CPU fallback:
+if the shared library is missing or a call fails, an exception is raised.
+PyTorch is used for device memory and streams only.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "lib", "libape.so")
+
+APE_PREFILL, APE_DECODE = 0, 1
+
+EXPORTS = ["ape_create", "ape_destroy", "ape_attend_plan", "ape_encode_plan", "ape_plan_workspace_bytes",
+           "ape_plan_destroy", "ape_attend", "ape_encode_contexts", "ape_attend_host", "ape_plan_last_launches",
+           "ape_get_status", "ape_status_string"]
+
+
+class ApeError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: libape status {code} ({status_string(code)})")
+        self.code = code
+
+
+class ape_shape_t(C.Structure):
+    _fields_ = [("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("softmax_scale", C.c_float)]
+
+
+class ape_span_t(C.Structure):
+    _fields_ = [("start", C.c_int64), ("len", C.c_int64)]
+
+
+class ape_kv_pool_t(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("n_tokens", C.c_int64), ("token_stride", C.c_int64), ("head_stride", C.c_int64)]
+
+
+class ape_rows_t(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("n_rows", C.c_int64), ("token_stride", C.c_int64), ("head_stride", C.c_int64)]
+
+
+class ape_request_t(C.Structure):
+    _fields_ = [("q_start", C.c_int64), ("q_len", C.c_int64), ("prefix", ape_span_t), ("ctx", C.POINTER(ape_span_t)),
+                ("n_ctx", C.c_int32), ("query_kv", ape_span_t), ("query_kv_capacity", C.c_int64)]
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Load libape.so (built in-tree by paper_2502_05431_b200.build).  Raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2502_05431_b200.build` "
+                              "(there is no fallback path)")
+        lib = C.CDLL(LIB_PATH)
+        vp = C.c_void_p
+        lib.ape_create.argtypes = [C.POINTER(vp), C.c_int]
+        lib.ape_destroy.argtypes = [vp]
+        lib.ape_attend_plan.argtypes = [vp, C.POINTER(ape_shape_t), C.POINTER(ape_kv_pool_t), C.POINTER(ape_rows_t),
+                                        C.POINTER(ape_rows_t), vp, C.POINTER(ape_request_t), C.c_int32, C.c_int, C.POINTER(vp)]
+        lib.ape_encode_plan.argtypes = [vp, C.POINTER(ape_shape_t), C.POINTER(ape_kv_pool_t), C.POINTER(ape_rows_t),
+                                        C.POINTER(ape_rows_t), vp, C.POINTER(ape_span_t), C.POINTER(ape_span_t), C.c_int32,
+                                        C.POINTER(vp)]
+        lib.ape_plan_workspace_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
+        lib.ape_plan_destroy.argtypes = [vp]
+        lib.ape_attend.argtypes = [vp, C.c_float, C.c_float, C.c_int64, vp, C.c_size_t, vp]
+        lib.ape_encode_contexts.argtypes = [vp, vp, C.c_size_t, vp]
+        lib.ape_attend_host.argtypes = [vp, C.c_float, C.c_float, C.c_int64, vp, C.c_size_t, vp, vp, vp, vp,
+                                        C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), vp]
+        lib.ape_plan_last_launches.argtypes = [vp, C.POINTER(C.c_int32)]
+        lib.ape_get_status.argtypes = [vp, C.POINTER(C.c_int32)]
+        lib.ape_status_string.argtypes = [C.c_int]
+        lib.ape_status_string.restype = C.c_char_p
+        for name in EXPORTS:
+            if name != "ape_status_string":
+                getattr(lib, name).restype = C.c_int
+        _lib = lib
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return load().ape_status_string(int(code)).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != 0:
+        raise ApeError(code, what)
+
+
+def _rows(t: torch.Tensor) -> ape_rows_t:
+    return ape_rows_t(t.data_ptr(), t.shape[0], t.stride(0), t.stride(1))
+
+
+def _pool(k: torch.Tensor, v: torch.Tensor) -> ape_kv_pool_t:
+    if k.shape != v.shape or k.stride() != v.stride():
+        raise ValueError("K and V pools must share shape and strides")
+    return ape_kv_pool_t(k.data_ptr(), v.data_ptr(), k.shape[0], k.stride(0), k.stride(1))
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+class Handle:
+    """ape_create / ape_destroy."""
+
+    def __init__(self, device: int = 0):
+        self._h = C.c_void_p()
+        _check(load().ape_create(C.byref(self._h), int(device)), "ape_create")
+        self.device = int(device)
+
+    def close(self) -> None:
+        if self._h:
+            load().ape_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def get_status(self) -> int:
+        v = C.c_int32(0)
+        _check(load().ape_get_status(self._h, C.byref(v)), "ape_get_status")
+        return int(v.value)
+
+    def attend_plan(self, *, H_q: int, H_kv: int, d: int, k_pool: torch.Tensor, v_pool: torch.Tensor,
+                    q: torch.Tensor, out: torch.Tensor, requests: Sequence, mode: int,
+                    lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0) -> "Plan":
+        """ape_attend_plan.  `requests`: objects with q_start, q_len, prefix, ctx, query_kv, query_kv_capacity
+        (spans are (start, len) pairs), e.g. paper_2502_05431_b200.workloads.Request."""
+        shape = ape_shape_t(H_q, H_kv, d, softmax_scale)
+        pool, qr, orows = _pool(k_pool, v_pool), _rows(q), _rows(out)
+        n = len(requests)
+        arr = (ape_request_t * max(n, 1))()
+        keep = []
+        for i, r in enumerate(requests):
+            spans = (ape_span_t * max(len(r.ctx), 1))(*[ape_span_t(int(s), int(l)) for s, l in r.ctx])
+            keep.append(spans)
+            arr[i] = ape_request_t(int(r.q_start), int(r.q_len), ape_span_t(*map(int, r.prefix)), spans, len(r.ctx),
+                                   ape_span_t(*map(int, r.query_kv)), int(r.query_kv_capacity))
+        p = C.c_void_p()
+        _check(load().ape_attend_plan(self._h, C.byref(shape), C.byref(pool), C.byref(qr), C.byref(orows),
+                                      lse.data_ptr() if lse is not None else None, arr, n, int(mode), C.byref(p)),
+               "ape_attend_plan")
+        return Plan(self, p, (q, out, k_pool, v_pool, lse))
+
+    def encode_plan(self, *, H_q: int, H_kv: int, d: int, k_pool: torch.Tensor, v_pool: torch.Tensor,
+                    q: torch.Tensor, out: torch.Tensor, prefix, ctx: Sequence,
+                    lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0) -> "Plan":
+        """ape_encode_plan.  q / out rows are aligned with the pool tokens."""
+        shape = ape_shape_t(H_q, H_kv, d, softmax_scale)
+        pool, qr, orows = _pool(k_pool, v_pool), _rows(q), _rows(out)
+        pre = ape_span_t(int(prefix[0]), int(prefix[1]))
+        spans = (ape_span_t * max(len(ctx), 1))(*[ape_span_t(int(s), int(l)) for s, l in ctx])
+        p = C.c_void_p()
+        _check(load().ape_encode_plan(self._h, C.byref(shape), C.byref(pool), C.byref(qr), C.byref(orows),
+                                      lse.data_ptr() if lse is not None else None, C.byref(pre), spans, len(ctx), C.byref(p)),
+               "ape_encode_plan")
+        return Plan(self, p, (q, out, k_pool, v_pool, lse))
+
+
+class Plan:
+    """An attend or encode plan: ape_plan_workspace_bytes / ape_attend / ape_encode_contexts / ape_plan_destroy."""
+
+    def __init__(self, handle: Handle, p: C.c_void_p, keep_alive):
+        self._handle, self._p, self._keep = handle, p, keep_alive
+        n = C.c_size_t(0)
+        _check(load().ape_plan_workspace_bytes(self._p, C.byref(n)), "ape_plan_workspace_bytes")
+        self.workspace_bytes = int(n.value)
+
+    def alloc_workspace(self, device=None) -> torch.Tensor:
+        dev = device if device is not None else self._keep[0].device
+        return torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=dev)
+
+    def attend(self, T: float, S: float, workspace: torch.Tensor, kv_extra: int = 0,
+               stream: Optional[torch.cuda.Stream] = None) -> None:
+        _check(load().ape_attend(self._p, float(T), float(S), int(kv_extra), workspace.data_ptr(), workspace.numel(),
+                                 _stream_ptr(stream)), "ape_attend")
+
+    def encode_contexts(self, workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> None:
+        _check(load().ape_encode_contexts(self._p, workspace.data_ptr() if workspace is not None else None,
+                                          workspace.numel() if workspace is not None else 0, _stream_ptr(stream)),
+               "ape_encode_contexts")
+
+    def attend_host(self, T: float, S: float, workspace: torch.Tensor, h_q: torch.Tensor, h_k: torch.Tensor,
+                    h_v: torch.Tensor, h_out: torch.Tensor, kv_extra: int = 0,
+                    stream: Optional[torch.cuda.Stream] = None):
+        """ape_attend_host: host tensors in, host tensor out; returns (h2d_bytes, d2h_bytes)."""
+        a, b = C.c_size_t(0), C.c_size_t(0)
+        _check(load().ape_attend_host(self._p, float(T), float(S), int(kv_extra), workspace.data_ptr(), workspace.numel(),
+                                      h_q.data_ptr(), h_k.data_ptr(), h_v.data_ptr(), h_out.data_ptr(),
+                                      C.byref(a), C.byref(b), _stream_ptr(stream)), "ape_attend_host")
+        return int(a.value), int(b.value)
+
+    def last_launches(self) -> int:
+        n = C.c_int32(0)
+        _check(load().ape_plan_last_launches(self._p, C.byref(n)), "ape_plan_last_launches")
+        return int(n.value)
+
+    def close(self) -> None:
+        if self._p:
+            load().ape_plan_destroy(self._p)
+            self._p = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

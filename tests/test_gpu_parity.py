@@ -1,0 +1,181 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle, element by element on the same
+seeded inputs.  Tolerance (bf16 output, fp32 accumulation): max-abs 2e-2, mean-abs 2e-3; relative L2 reported."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ape_oracle as orc
+from paper_2502_05431_b200 import libape
+from paper_2502_05431_b200 import workloads as wl
+from tests.gpu_util import compare, gpu_attend, handle, oracle_attend
+
+pytestmark = pytest.mark.gpu
+LLAMA = dict(H_q=32, H_kv=8, d=128)
+
+
+def _check_batch(b, mode, rows=None, lse_tol=2e-3, **kw):
+    out, lse, n = gpu_attend(b, mode, **kw)
+    assert n == 2
+    for r, rq in enumerate(b.requests):
+        ref = oracle_attend(b, r, rows=rows, l_k=(rq.query_kv[1] + kw.get("kv_extra", 0)) if kw.get("kv_extra") else None,
+                            q_override=None if kw.get("q_override") is None else kw["q_override"][rq.q_start:rq.q_start + rq.q_len])
+        compare(out[rq.q_start:rq.q_start + rq.q_len], ref.out.float(), f"{b.name} req {r} O")
+        sel = ~torch.isnan(ref.lse)
+        d = (lse[rq.q_start:rq.q_start + rq.q_len].double()[sel] - ref.lse[sel]).abs().max().item()
+        assert d < lse_tol, f"{b.name} req {r}: LSE error {d}"
+
+
+# ---- decode -------------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("kw", [
+    dict(H_q=4, H_kv=1, d=64, l_P=16, ctx_lens=[[64] * 4], l_k=17, T=0.8, S=0.9),                  # tiny, d = 64
+    dict(**LLAMA, l_P=5, ctx_lens=[[70, 1, 129], [200]], l_k=3, gap=3, T=0.7, S=0.8),               # ragged, gaps, 2 requests
+    dict(**LLAMA, l_P=0, ctx_lens=[[]], l_k=1),                                                      # only its own key
+    dict(**LLAMA, l_P=0, ctx_lens=[[333]], l_k=1, T=0.5, S=1.2, shuffle_ctx=True),
+    dict(H_q=16, H_kv=1, d=128, l_P=64, ctx_lens=[[256] * 3], l_k=65, T=0.9, S=0.9),                # G = 16
+    dict(H_q=8, H_kv=8, d=64, l_P=3, ctx_lens=[[100, 100]], l_k=9, T=0.9, S=0.5),                   # G = 1
+])
+def test_decode_small(kw):
+    b = wl.make_batch(l_q=1, seed=1, name="decode_small", **kw)
+    _check_batch(b, libape.APE_DECODE)
+
+
+def test_decode_many_tiles_and_growing_query_segment():
+    """Enough tokens that every CTA holds several items; kv_extra grows the query segment step by step."""
+    b = wl.make_batch(**LLAMA, l_P=64, ctx_lens=[[256] * 40, [512] * 11], l_q=1, l_k=100, capacity=100 + 70, seed=2,
+                      T=0.9, S=0.9, name="decode_grow")
+    for t in (0, 1, 27, 70):
+        _check_batch(b, libape.APE_DECODE, kv_extra=t)
+
+
+def test_decode_rejects_bad_arguments():
+    b = wl.make_batch(**LLAMA, l_P=8, ctx_lens=[[64]], l_q=1, l_k=4, capacity=6, seed=3)
+    dev = torch.device("cuda:0")
+    q, k, v = b.q.to(dev), b.k_pool.to(dev), b.v_pool.to(dev)
+    out = torch.empty_like(q)
+    plan = handle().attend_plan(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=q, out=out, requests=b.requests, mode=libape.APE_DECODE)
+    ws = plan.alloc_workspace()
+    for T, S in [(0.0, 1.0), (1.0, -1.0), (float("nan"), 1.0), (1.0, float("inf"))]:
+        with pytest.raises(libape.ApeError) as e:
+            plan.attend(T, S, ws)
+        assert e.value.code == -4
+    with pytest.raises(libape.ApeError) as e:
+        plan.attend(1.0, 1.0, ws, kv_extra=3)          # beyond the reserved capacity
+    assert e.value.code == -4
+    with pytest.raises(libape.ApeError) as e:
+        plan.attend(1.0, 1.0, ws[:256])                # workspace too small
+    assert e.value.code == -6
+    with pytest.raises(libape.ApeError) as e:
+        plan.encode_contexts()
+    assert e.value.code == -10
+    with pytest.raises(libape.ApeError) as e:          # head_dim 96 unsupported
+        handle().attend_plan(H_q=32, H_kv=8, d=96, k_pool=k, v_pool=v, q=q, out=out, requests=b.requests, mode=libape.APE_DECODE)
+    assert e.value.code == -2
+    bad = wl.Request(0, 1, (0, 8), [(10, 10 ** 9)], b.requests[0].query_kv, 6)
+    with pytest.raises(libape.ApeError) as e:
+        handle().attend_plan(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=q, out=out, requests=[bad], mode=libape.APE_DECODE)
+    assert e.value.code == -1
+
+
+# ---- query prefill ----------------------------------------------------------------------------------------------------
+
+def test_prefill_config1_tiny():
+    _check_batch(wl.config1(), libape.APE_PREFILL)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(**LLAMA, l_P=32, ctx_lens=[[256] * 10], l_q=64, T=0.9, S=0.9),                     # config 2
+    dict(**LLAMA, l_P=7, ctx_lens=[[130, 1, 255], [77]], l_q=33, l_k=50, gap=5, T=0.6, S=0.7),    # ragged, l_k > l_q
+    dict(**LLAMA, l_P=0, ctx_lens=[[]], l_q=200, T=1.0, S=1.0),                             # plain causal attention
+    dict(H_q=8, H_kv=8, d=64, l_P=10, ctx_lens=[[300]], l_q=300, T=0.8, S=1.1),             # G = 1, d = 64, 2 row blocks
+    dict(H_q=16, H_kv=1, d=128, l_P=64, ctx_lens=[[256] * 4], l_q=40, T=0.9, S=0.9),        # G = 16
+    dict(**LLAMA, l_P=64, ctx_lens=[[512] * 9], l_q=320, T=0.9, S=0.9),                     # 5 row blocks > 4 siblings
+])
+def test_prefill_shapes(kw):
+    b = wl.make_batch(seed=4, name="prefill", **kw)
+    _check_batch(b, libape.APE_PREFILL)
+
+
+def test_prefill_ignores_garbage_outside_spans():
+    """Pool tokens that belong to no span (gaps, reserved capacity) may hold NaN without affecting the result."""
+    b = wl.make_batch(**LLAMA, l_P=20, ctx_lens=[[100, 60]], l_q=16, l_k=16, capacity=40, gap=7, seed=5, T=0.8, S=0.9, name="garbage")
+    used = torch.zeros(b.k_pool.shape[0], dtype=torch.bool)
+    rq = b.requests[0]
+    for s, n in [rq.prefix, rq.query_kv] + rq.ctx:
+        used[s:s + n] = True
+    b.k_pool[~used] = float("nan")
+    b.v_pool[~used] = float("nan")
+    _check_batch(b, libape.APE_PREFILL)
+    b1 = wl.make_batch(**LLAMA, l_P=20, ctx_lens=[[100, 60]], l_q=1, l_k=16, capacity=40, gap=7, seed=5, T=0.8, S=0.9, name="garbage_dec")
+    b1.k_pool[~used] = float("nan")
+    b1.v_pool[~used] = float("nan")
+    _check_batch(b1, libape.APE_DECODE)
+
+
+@pytest.mark.parametrize("T,S", [(0.5, 0.8), (0.5, 1.0), (0.9, 0.8), (0.9, 1.0)])
+def test_prefill_config3_rag(T, S):
+    b = wl.config3(T=T, S=S)
+    out, lse, _ = gpu_attend(b, libape.APE_PREFILL)
+    for r, rq in enumerate(b.requests):
+        for rows in [(0, 4), (62, 66), (124, 128)]:
+            ref = oracle_attend(b, r, rows=rows)
+            compare(out[rq.q_start:rq.q_start + rq.q_len], ref.out.float(), f"cfg3 T={T} S={S} req {r} rows {rows}")
+
+
+def test_prefill_config4_manyshot_128k_sampled_rows():
+    b = wl.config4()
+    out, lse, _ = gpu_attend(b, libape.APE_PREFILL)
+    assert not torch.isnan(out.float()).any()
+    for rows in [(0, 2), (127, 129), (254, 256)]:
+        ref = oracle_attend(b, 0, rows=rows)
+        compare(out, ref.out.float(), f"cfg4 rows {rows}")
+        sel = ~torch.isnan(ref.lse)
+        assert (lse.double()[sel] - ref.lse[sel]).abs().max().item() < 2e-3
+
+
+def test_decode_config5_128k_sampled_requests():
+    b = wl.config5(n_req=16)
+    dev = torch.device("cuda:0")
+    q_steps = b.extra["q_steps"]
+    for t in (0, 128, 255):
+        out, lse, _ = gpu_attend(b, libape.APE_DECODE, kv_extra=t, q_override=q_steps[t].contiguous())
+        for r in (0, 7, 15):
+            ref = oracle_attend(b, r, l_k=257 + t, q_override=q_steps[t, r:r + 1].contiguous())
+            compare(out[r:r + 1], ref.out.float(), f"cfg5 step {t} req {r}")
+
+
+# ---- encode -----------------------------------------------------------------------------------------------------------
+
+def _check_encode(b):
+    dev = torch.device("cuda:0")
+    q, k, v = b.q_enc.to(dev), b.k_pool.to(dev), b.v_pool.to(dev)
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((q.shape[0], b.H_q), float("nan"), dtype=torch.float32, device=dev)
+    rq = b.requests[0]
+    plan = handle().encode_plan(H_q=b.H_q, H_kv=b.H_kv, d=b.d, k_pool=k, v_pool=v, q=q, out=out, prefix=rq.prefix, ctx=rq.ctx, lse=lse)
+    plan.encode_contexts()
+    torch.cuda.synchronize()
+    assert handle().get_status() == 0
+    out, lse = out.cpu(), lse.cpu()
+    _, p, c, _ = b.views(0)
+    qs = [b.q_enc[s:s + n] for s, n in rq.ctx]
+    refs, lses = orc.encode(qs, p, c)
+    touched = torch.zeros(out.shape[0], dtype=torch.bool)
+    for (s, n), ref, l in zip(rq.ctx, refs, lses):
+        if n == 0:
+            continue
+        compare(out[s:s + n], ref.float(), f"{b.name} ctx@{s}")
+        assert (lse[s:s + n].double() - l).abs().max().item() < 2e-3
+        touched[s:s + n] = True
+    assert torch.isnan(out[~touched].float()).all(), "rows outside the context spans were written"
+
+
+@pytest.mark.parametrize("kw", [
+    dict(H_q=4, H_kv=1, d=64, l_P=16, ctx_lens=[[64] * 4]),                        # config 1 shape
+    dict(**LLAMA, l_P=32, ctx_lens=[[256] * 10]),                                  # config 2
+    dict(**LLAMA, l_P=0, ctx_lens=[[1, 129, 0, 300]], gap=3),                      # ragged, no prefix, an empty context
+    dict(**LLAMA, l_P=200, ctx_lens=[[70, 700]]),                                  # prefix longer than a tile; 11 row blocks
+])
+def test_encode(kw):
+    b = wl.make_batch(l_q=1, seed=6, with_encode_q=True, name="encode", **kw)
+    _check_encode(b)
