@@ -63,7 +63,7 @@ class Batch:
 
 
 def _randn_bf16(gen: torch.Generator, shape, scale: Optional[torch.Tensor] = None) -> torch.Tensor:
-    x = torch.randn(shape, generator=gen, dtype=torch.float32)
+    x = torch.randn(shape, generator=gen, dtype=torch.float32, device=gen.device)
     if scale is not None:
         x = x * scale.view(1, -1, 1)
     return x.to(torch.bfloat16)
@@ -72,32 +72,36 @@ def _randn_bf16(gen: torch.Generator, shape, scale: Optional[torch.Tensor] = Non
 def make_batch(*, H_q: int, H_kv: int, d: int, l_P: int, ctx_lens: Sequence[Sequence[int]], l_q: int,
                l_k: Optional[int] = None, capacity: Optional[int] = None, seed: int = 0,
                T: float = 1.0, S: float = 1.0, head_scale: bool = False, gap: int = 0,
-               with_encode_q: bool = False, shuffle_ctx: bool = False, name: str = "") -> Batch:
+               with_encode_q: bool = False, shuffle_ctx: bool = False, name: str = "",
+               device: Optional[str] = None) -> Batch:
     """Build a batch of ``len(ctx_lens)`` requests with independent context sets.
 
     ``gap`` leaves that many unused (zero) tokens after every span so that spans are
     not adjacent; ``shuffle_ctx`` lists each request's contexts in a seeded random
     order different from their order in the pool.  ``l_k`` is the number of keys in the
     query's own segment (default ``l_q``); ``capacity`` reserves room for decode appends.
+    ``device``: draw and keep the tensors there (e.g. "cuda:0", for workloads too large to draw on the host
+    in reasonable time); the values then come from that device's generator, same distribution and layout.
     """
+    dev = torch.device(device) if device is not None else torch.device("cpu")
     n_req = len(ctx_lens)
     l_k = l_q if l_k is None else l_k
     capacity = l_k if capacity is None else capacity
     assert capacity >= l_k >= l_q
     per_req_tokens = [l_P + sum(cl) + capacity + gap * (len(cl) + 2) for cl in ctx_lens]
     pool_tokens = sum(per_req_tokens)
-    k_pool = torch.zeros((pool_tokens, H_kv, d), dtype=torch.bfloat16)
-    v_pool = torch.zeros((pool_tokens, H_kv, d), dtype=torch.bfloat16)
-    q = torch.zeros((n_req * l_q, H_q, d), dtype=torch.bfloat16)
-    q_enc = torch.zeros((pool_tokens, H_q, d), dtype=torch.bfloat16) if with_encode_q else None
+    k_pool = torch.zeros((pool_tokens, H_kv, d), dtype=torch.bfloat16, device=dev)
+    v_pool = torch.zeros((pool_tokens, H_kv, d), dtype=torch.bfloat16, device=dev)
+    q = torch.zeros((n_req * l_q, H_q, d), dtype=torch.bfloat16, device=dev)
+    q_enc = torch.zeros((pool_tokens, H_q, d), dtype=torch.bfloat16, device=dev) if with_encode_q else None
     requests: List[Request] = []
     cur = 0
     for r, lens in enumerate(ctx_lens):
-        gen = torch.Generator(device="cpu").manual_seed(seed + r)
+        gen = torch.Generator(device=dev).manual_seed(seed + r)
         sk = sv = None
         if head_scale:
-            sk = torch.rand(H_kv, generator=gen) * 1.5 + 0.5
-            sv = torch.rand(H_kv, generator=gen) * 1.5 + 0.5
+            sk = torch.rand(H_kv, generator=gen, device=dev) * 1.5 + 0.5
+            sv = torch.rand(H_kv, generator=gen, device=dev) * 1.5 + 0.5
         q[r * l_q:(r + 1) * l_q] = _randn_bf16(gen, (l_q, H_q, d))
         prefix = (cur, l_P)
         if l_P:
@@ -120,7 +124,7 @@ def make_batch(*, H_q: int, H_kv: int, d: int, l_P: int, ctx_lens: Sequence[Sequ
                 if L:
                     q_enc[s:s + L] = _randn_bf16(gen, (L, H_q, d))
         if shuffle_ctx and len(spans) > 1:
-            perm = torch.randperm(len(spans), generator=gen).tolist()
+            perm = torch.randperm(len(spans), generator=gen, device=dev).tolist()
             spans = [spans[p] for p in perm]
         requests.append(Request(r * l_q, l_q, prefix, spans, qkv, capacity))
     assert cur == pool_tokens
@@ -155,13 +159,13 @@ def config3(seed: int = 0, T: float = 0.9, S: float = 0.8) -> Batch:
                       name="cfg3_rag")
 
 
-def config4(seed: int = 0, n_ctx: int = 500) -> Batch:
+def config4(seed: int = 0, n_ctx: int = 500, with_encode_q: bool = False, device: Optional[str] = None) -> Batch:
     """Many-shot 128K: prefix 64, 500 contexts x 256 tokens, 256 causal query rows, per-KV-head scale U[0.5,2]."""
     return make_batch(**LLAMA3_8B, l_P=64, ctx_lens=[[256] * n_ctx], l_q=256, seed=seed, T=0.9, S=0.9,
-                      head_scale=True, name="cfg4_manyshot_128k")
+                      head_scale=True, with_encode_q=with_encode_q, name="cfg4_manyshot_128k", device=device)
 
 
-def config5(seed: int = 0, n_req: int = 16, n_ctx: int = 500, steps: int = 256) -> Batch:
+def config5(seed: int = 0, n_req: int = 16, n_ctx: int = 500, steps: int = 256, device: Optional[str] = None) -> Batch:
     """Decode at 128K: per request prefix 64 + 500x256 contexts + 256 cached query tokens; one new row per step.
 
     The pool reserves ``256 + steps`` query-segment tokens per request, all pre-drawn, so step t reads
@@ -169,8 +173,9 @@ def config5(seed: int = 0, n_req: int = 16, n_ctx: int = 500, steps: int = 256) 
     bf16 ``[steps, n_req, H_q, d]``.
     """
     b = make_batch(**LLAMA3_8B, l_P=64, ctx_lens=[[256] * n_ctx] * n_req, l_q=1, l_k=257, capacity=256 + steps,
-                   seed=seed, T=0.9, S=0.9, name="cfg5_decode_128k")
-    gen = torch.Generator(device="cpu").manual_seed(seed + 7919)
-    b.extra["q_steps"] = torch.randn((steps, n_req, b.H_q, b.d), generator=gen, dtype=torch.float32).to(torch.bfloat16)
+                   seed=seed, T=0.9, S=0.9, name="cfg5_decode_128k", device=device)
+    gen = torch.Generator(device=b.q.device).manual_seed(seed + 7919)
+    b.extra["q_steps"] = torch.randn((steps, n_req, b.H_q, b.d), generator=gen, dtype=torch.float32,
+                                     device=b.q.device).to(torch.bfloat16)
     b.extra["steps"] = steps
     return b
