@@ -332,9 +332,17 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     #pragma unroll
                     for (int i = 0; i < kTileN; ++i) s[i] = (i < limit) ? s[i] : -INFINITY;
                 }
-                float mx = s[0];
+                // eight independent running maxima keep the dependency chain short
+                float mxa[8];
                 #pragma unroll
-                for (int i = 1; i < kTileN; ++i) mx = fmaxf(mx, s[i]);
+                for (int k = 0; k < 8; ++k) mxa[k] = s[k];
+                #pragma unroll
+                for (int i = 8; i < kTileN; i += 8) {
+                    #pragma unroll
+                    for (int k = 0; k < 8; ++k) mxa[k] = fmaxf(mxa[k], s[i + k]);
+                }
+                const float mx = fmaxf(fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])),
+                                       fmaxf(fmaxf(mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
                 const float m_new = fmaxf(m, mx * scale);
                 if (n_local == 0) {
                     m = m_new;
@@ -359,7 +367,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
                 const float m_use = (m == -INFINITY) ? 0.f : m;
-                float sum = 0.f;
+                float sum[4] = {0.f, 0.f, 0.f, 0.f};
                 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     uint32_t pk[32];
@@ -367,12 +375,12 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     for (int i = 0; i < 32; ++i) {
                         const float p0 = fast_exp2(fmaf(s[hh * 64 + 2 * i], scale, -m_use));
                         const float p1 = fast_exp2(fmaf(s[hh * 64 + 2 * i + 1], scale, -m_use));
-                        sum += p0 + p1;
+                        sum[i & 3] += p0 + p1;
                         pk[i] = pack_bf16x2(p0, p1);
                     }
                     tmem_st32(tS + hh * 32, pk);
                 }
-                l += sum;
+                l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
                 tmem_st_wait();
                 tc_fence_before();
                 mbar_arrive(my_p_full);

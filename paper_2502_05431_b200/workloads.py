@@ -103,23 +103,31 @@ def make_batch(*, H_q: int, H_kv: int, d: int, l_P: int, ctx_lens: Sequence[Sequ
             sk = torch.rand(H_kv, generator=gen, device=dev) * 1.5 + 0.5
             sv = torch.rand(H_kv, generator=gen, device=dev) * 1.5 + 0.5
         q[r * l_q:(r + 1) * l_q] = _randn_bf16(gen, (l_q, H_q, d))
+        bulk = dev.type != "cpu"     # on a device: one draw per tensor and request (same distribution, few launches)
+        if bulk:
+            n_tok = per_req_tokens[r]
+            k_pool[cur:cur + n_tok] = _randn_bf16(gen, (n_tok, H_kv, d), sk)
+            v_pool[cur:cur + n_tok] = _randn_bf16(gen, (n_tok, H_kv, d), sv)
+            if with_encode_q:
+                q_enc[cur:cur + n_tok] = _randn_bf16(gen, (n_tok, H_q, d))
         prefix = (cur, l_P)
-        if l_P:
+        if l_P and not bulk:
             k_pool[cur:cur + l_P] = _randn_bf16(gen, (l_P, H_kv, d), sk)
             v_pool[cur:cur + l_P] = _randn_bf16(gen, (l_P, H_kv, d), sv)
         cur += l_P + gap
         spans: List[Span] = []
         for L in lens:
-            if L:
+            if L and not bulk:
                 k_pool[cur:cur + L] = _randn_bf16(gen, (L, H_kv, d), sk)
                 v_pool[cur:cur + L] = _randn_bf16(gen, (L, H_kv, d), sv)
             spans.append((cur, L))
             cur += L + gap
         qkv = (cur, l_k)
-        k_pool[cur:cur + capacity] = _randn_bf16(gen, (capacity, H_kv, d), sk)
-        v_pool[cur:cur + capacity] = _randn_bf16(gen, (capacity, H_kv, d), sv)
+        if not bulk:
+            k_pool[cur:cur + capacity] = _randn_bf16(gen, (capacity, H_kv, d), sk)
+            v_pool[cur:cur + capacity] = _randn_bf16(gen, (capacity, H_kv, d), sv)
         cur += capacity + gap
-        if with_encode_q:
+        if with_encode_q and not bulk:
             for (s, L) in spans:
                 if L:
                     q_enc[s:s + L] = _randn_bf16(gen, (L, H_q, d))
