@@ -137,6 +137,39 @@ int ape_attend_host(ape_plan_t plan, float T, float S, int64_t kv_extra, void *w
                     const void *h_q, const void *h_k_pool, const void *h_v_pool, void *h_out,
                     size_t *h2d_bytes, size_t *d2h_bytes, void *stream);
 
+/*
+ * Allocation-free decode step.  (The paper has no counterpart to this entry point; it exists for the callers
+ * described here.)  Some hosts of this library must not allocate device memory at call time: an inference server
+ * that has handed the whole GPU to its own memory pool (a cudaMalloc there fails or fragments the pool), a
+ * latency-critical decode loop that cannot afford the device-wide synchronisation an allocation may imply, or a
+ * plug-in that runs under a policy forbidding the allocator.  ape_create and the plan calls above allocate (status
+ * word, plan metadata) and take a caller-provided workspace; this call needs none of them.  It computes exactly
+ * what an APE_DECODE plan followed by ape_attend computes (one query row per request, Eq. 5), with the same kernels,
+ * but keeps the plan metadata, the split-KV partials and the status word in a fixed 8 MiB device array that is
+ * part of the library image.  Every GPU that loads the library holds those 8 MiB until the process exits.
+ *
+ *   - Arguments as in ape_attend_plan (mode APE_DECODE) and ape_attend; `device` is the CUDA ordinal the tensors
+ *     live on; `lse` is nullable.  The caller still owns and passes every input and output tensor.
+ *   - Limits: the tile lists and work items of the batch must fit 4 MiB and the partials the other 4 MiB
+ *     (roughly: up to ~250,000 64-token tiles over all requests, i.e. about 16M cached tokens, and
+ *     (SMs + 2 * n_req * H_kv) * (H_q / H_kv) * d * 4 bytes of partials).  A larger batch is rejected with
+ *     APE_ERR_WORKSPACE before anything is launched; nothing is ever allocated instead.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and the device's
+ *     properties; make that first call outside any stream capture.  With lazy module loading this lookup is also
+ *     the moment the runtime materialises the array, so the driver's free-memory figure drops by 8 MiB once.  Later calls only do host work, two
+ *     stream-ordered copies/memsets into the array and two kernel launches on `stream`.
+ *   - Calls no cudaMalloc, cudaFree, or any other allocating routine.  Host descriptors are read during the call.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents: each call rewrites
+ *     the metadata it uses and clears the status word first.  Two calls whose GPU work may overlap (different
+ *     streams, or different threads) race on the array: order them on one stream or with events.
+ *   - Asynchronous like ape_attend when `device_status` is NULL.  With a non-NULL `device_status` (HOST pointer)
+ *     the call synchronises `stream` after its launches and stores the array's status word there: 0, or
+ *     APE_ERR_TIMEOUT if a kernel gave up on a bounded wait.
+ */
+int ape_decode_noalloc(const ape_shape_t *shape, const ape_kv_pool_t *pool, const ape_rows_t *q,
+                       const ape_rows_t *out, float *lse, const ape_request_t *requests, int32_t n_req,
+                       float T, float S, int64_t kv_extra, int device, void *stream, int32_t *device_status);
+
 /* Kernels launched by the last ape_attend / ape_encode_contexts call on this plan. */
 int ape_plan_last_launches(ape_plan_t plan, int32_t *n_launches);
 

@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -568,6 +569,177 @@ const char* ape_status_string(int s) {
         case APE_ERR_MODE: return "plan used with the wrong entry point";
         default: return "unknown status";
     }
+}
+
+}  // extern "C"
+
+// ---- allocation-free decode ------------------------------------------------------------------------------------------
+// A decode step for callers that must not allocate device memory (see include/ape.h).  Everything a plan would put
+// into cudaMalloc'ed memory or into the caller's workspace lives in one fixed device array of the library image.
+
+namespace {
+
+constexpr size_t kNoAllocBytes = 8u << 20;        // whole array
+constexpr size_t kNoAllocMetaBytes = 4u << 20;    // [0, 256): status word; then tiles, items, CTA ranges, requests, merge groups
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+struct NoAllocDevice {
+    bool ready = false;
+    unsigned char* scratch = nullptr;             // DEVICE address of g_noalloc_scratch on this device
+    ape_handle_s h;                               // host-side record only (no device allocation behind it)
+};
+constexpr int kMaxDevices = 64;
+NoAllocDevice g_noalloc_dev[kMaxDevices];
+std::mutex g_noalloc_mutex;
+
+// Once per device, with that device current: the array's name is a host-side stand-in here, so ask the runtime for
+// the address the kernels must be given.
+int noalloc_setup(int device, NoAllocDevice** out) {
+    if (device < 0 || device >= kMaxDevices) return APE_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    NoAllocDevice& d = g_noalloc_dev[device];
+    if (cudaSetDevice(device) != cudaSuccess) return APE_ERR_CUDA;
+    if (!d.ready) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return APE_ERR_CUDA;
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return APE_ERR_CUDA;
+        if (prop.major != 10) return APE_ERR_CUDA;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) return APE_ERR_CUDA;
+        d.scratch = static_cast<unsigned char*>(ptr);
+        d.h.device = device; d.h.n_sm = prop.multiProcessorCount; d.h.smem_optin = prop.sharedMemPerBlockOptin;
+        d.h.d_status = reinterpret_cast<int*>(d.scratch);
+        d.h.encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+        d.ready = true;
+    }
+    *out = &d;
+    return APE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q, const ape_rows_t* out,
+                       float* lse, const ape_request_t* reqs, int32_t n_req, float T, float S, int64_t kv_extra,
+                       int device, void* stream_v, int32_t* device_status)
+{
+    int G = 1; float c = 0.f;
+    int rc = check_shape(shape, &G, &c);              if (rc) return rc;
+    rc = check_pool(pool, shape);                     if (rc) return rc;
+    rc = check_rows(q, shape);                        if (rc) return rc;
+    rc = check_rows(out, shape);                      if (rc) return rc;
+    if (!reqs || n_req <= 0 || out->n_rows < q->n_rows) return APE_ERR_INVALID_ARG;
+    if (!(T > 0.f) || !(S > 0.f) || !std::isfinite(T) || !std::isfinite(S)) return APE_ERR_RANGE;
+    int64_t max_extra = INT64_MAX, total_tiles = 0;
+    for (int r = 0; r < n_req; ++r) {
+        const ape_request_t& rq = reqs[r];
+        if (rq.q_len != 1 || rq.q_start < 0 || rq.q_start + 1 > q->n_rows) return APE_ERR_INVALID_ARG;
+        if (rq.n_ctx < 0 || (rq.n_ctx > 0 && !rq.ctx)) return APE_ERR_INVALID_ARG;
+        if (!span_ok(rq.prefix, pool->n_tokens) || !span_ok(rq.query_kv, pool->n_tokens)) return APE_ERR_INVALID_ARG;
+        if (rq.query_kv.len < 1) return APE_ERR_INVALID_ARG;
+        if (rq.query_kv_capacity < rq.query_kv.len || rq.query_kv.start + rq.query_kv_capacity > pool->n_tokens) return APE_ERR_INVALID_ARG;
+        total_tiles += (rq.prefix.len + kDecodeTile - 1) / kDecodeTile + (rq.query_kv_capacity + kDecodeTile - 1) / kDecodeTile;
+        for (int i = 0; i < rq.n_ctx; ++i) {
+            if (!span_ok(rq.ctx[i], pool->n_tokens)) return APE_ERR_INVALID_ARG;
+            total_tiles += (rq.ctx[i].len + kDecodeTile - 1) / kDecodeTile;
+        }
+        max_extra = std::min(max_extra, rq.query_kv_capacity - rq.query_kv.len);
+    }
+    if (kv_extra < 0 || kv_extra > max_extra) return APE_ERR_RANGE;
+    // size gate, before any host vector grows and before anything touches the device
+    if (static_cast<size_t>(total_tiles) * sizeof(DevTile) > kNoAllocMetaBytes) return APE_ERR_WORKSPACE;
+
+    NoAllocDevice* dv = nullptr;
+    rc = noalloc_setup(device, &dv);                  if (rc) return rc;
+    const int D = shape->head_dim, H_kv = shape->n_kv_heads, tile = kDecodeTile;
+    const int n_cta = dv->h.n_sm;
+
+    HostMeta m;
+    std::vector<uint8_t> blob;
+    size_t o_tiles = 0, o_items = 0, o_cta = 0, o_reqs = 0, o_merge = 0;
+    try {
+        std::vector<Run> runs;
+        for (int r = 0; r < n_req; ++r) {
+            const ape_request_t& rq = reqs[r];
+            m.reqs.push_back(DevReq{static_cast<int32_t>(rq.q_start), 1, static_cast<int32_t>(rq.query_kv.len), 0});
+            const int o0 = static_cast<int>(m.tiles.size());
+            add_span_tiles(m.tiles, rq.prefix.start, rq.prefix.len, tile, 0, 0);
+            add_span_tiles(m.tiles, rq.query_kv.start, rq.query_kv.len, tile, TILE_GROWS, rq.query_kv_capacity);
+            const int o1 = static_cast<int>(m.tiles.size());
+            for (const auto& sp : fuse_spans(rq.ctx, rq.n_ctx)) add_span_tiles(m.tiles, sp.start, sp.len, tile, 0, 0);
+            const int c1 = static_cast<int>(m.tiles.size());
+            for (int hh = 0; hh < H_kv; ++hh) {
+                const int mi = static_cast<int>(m.merge.size());
+                m.merge.push_back(DevMerge{r, hh, 0, 0, 0, 0, 0, 1});
+                runs.push_back(Run{r, hh, 0, 1, SEG_OTHER, o0, o1, mi});
+                if (c1 > o1) runs.push_back(Run{r, hh, 0, 1, SEG_CTX, o1, c1, mi});
+            }
+        }
+        assign_stream(runs, n_cta, 1, m);
+        auto rnd = [](size_t x) { return (x + 255) & ~size_t(255); };
+        o_tiles = 256;                                                     // after the status word
+        o_items = o_tiles + rnd(m.tiles.size() * sizeof(DevTile));
+        o_cta = o_items + rnd(m.items.size() * sizeof(DevItem));
+        o_reqs = o_cta + rnd(m.cta_begin.size() * 4);
+        o_merge = o_reqs + rnd(m.reqs.size() * sizeof(DevReq));
+        const size_t meta_end = o_merge + rnd(m.merge.size() * sizeof(DevMerge));
+        const size_t rows = m.items.size() * static_cast<size_t>(G);
+        const size_t part_bytes = rnd(rows * D * 4) + rnd(rows * 2 * 4);
+        if (meta_end > kNoAllocMetaBytes || part_bytes > kNoAllocBytes - kNoAllocMetaBytes) return APE_ERR_WORKSPACE;
+        blob.assign(meta_end, 0);                                          // byte 0..255: the status word, cleared
+        std::memcpy(blob.data() + o_tiles, m.tiles.data(), m.tiles.size() * sizeof(DevTile));
+        std::memcpy(blob.data() + o_items, m.items.data(), m.items.size() * sizeof(DevItem));
+        std::memcpy(blob.data() + o_cta, m.cta_begin.data(), m.cta_begin.size() * 4);
+        std::memcpy(blob.data() + o_reqs, m.reqs.data(), m.reqs.size() * sizeof(DevReq));
+        std::memcpy(blob.data() + o_merge, m.merge.data(), m.merge.size() * sizeof(DevMerge));
+    } catch (const std::bad_alloc&) {
+        return APE_ERR_NOMEM;
+    }
+
+    const int n_stages = decode_pick_stages(D, G, dv->h.smem_optin - 2048);
+    if (n_stages < 2) return APE_ERR_SHAPE;
+    const size_t smem_bytes = decode_smem_bytes(D, G, n_stages);
+    if (decode_set_smem_attr(D, smem_bytes) != cudaSuccess) return APE_ERR_CUDA;
+    CUtensorMap tm_k, tm_v;
+    rc = make_map(&dv->h, &tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
+    if (!rc) rc = make_map(&dv->h, &tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
+    if (rc) return rc;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    unsigned char* base = dv->scratch;
+    // The array still holds the previous call's status word, metadata and partials.  The copy below rewrites the
+    // status word (zero) and all metadata this call uses; partial slots are fully written by the decode kernel before
+    // the merge kernel reads them, so they need no clearing.  The source is pageable host memory: the runtime has
+    // taken its copy of it when cudaMemcpyAsync returns.
+    if (cudaMemcpyAsync(base, blob.data(), blob.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess) return APE_ERR_CUDA;
+
+    constexpr float kLog2e = 1.4426950408889634f;
+    const size_t rows = m.items.size() * static_cast<size_t>(G);
+    float* ws_o = reinterpret_cast<float*>(base + kNoAllocMetaBytes);
+    float* ws_ml = reinterpret_cast<float*>(base + kNoAllocMetaBytes + ((rows * D * 4 + 255) & ~size_t(255)));
+    DecodeParams dp;
+    dp.tiles = reinterpret_cast<const DevTile*>(base + o_tiles); dp.items = reinterpret_cast<const DevItem*>(base + o_items);
+    dp.cta_item_begin = reinterpret_cast<const int32_t*>(base + o_cta); dp.reqs = reinterpret_cast<const DevReq*>(base + o_reqs);
+    dp.q = rows_desc(*q); dp.ws_o = ws_o; dp.ws_ml = ws_ml;
+    dp.scale_oth_log2 = c * kLog2e; dp.scale_ctx_log2 = c / T * kLog2e;
+    dp.kv_extra = static_cast<int32_t>(kv_extra); dp.G = G; dp.n_stages = n_stages; dp.status = reinterpret_cast<int*>(base);
+    if (launch_decode(D, tm_k, tm_v, dp, n_cta, smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
+    MergeParams mp;
+    mp.groups = reinterpret_cast<const DevMerge*>(base + o_merge); mp.reqs = dp.reqs; mp.n_groups = static_cast<int32_t>(m.merge.size());
+    mp.rows_per_slot = G; mp.tokens_per_block = 1; mp.ws_o = ws_o; mp.ws_ml = ws_ml; mp.out = rows_desc(*out); mp.lse_out = lse;
+    mp.S = S; mp.G = G; mp.H_q = shape->n_q_heads; mp.D = D;
+    if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;
+    if (device_status != nullptr) {
+        // the caller asked for the status word: this makes the call synchronous
+        int v = 0;
+        if (cudaMemcpyAsync(&v, base, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return APE_ERR_CUDA;
+        if (cudaStreamSynchronize(stream) != cudaSuccess) return APE_ERR_CUDA;
+        *device_status = v;
+    }
+    return APE_OK;
 }
 
 }  // extern "C"

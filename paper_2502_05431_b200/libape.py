@@ -19,7 +19,7 @@ APE_PREFILL, APE_DECODE = 0, 1
 
 EXPORTS = ["ape_create", "ape_destroy", "ape_attend_plan", "ape_encode_plan", "ape_plan_workspace_bytes",
            "ape_plan_destroy", "ape_attend", "ape_encode_contexts", "ape_attend_host", "ape_plan_last_launches",
-           "ape_get_status", "ape_status_string"]
+           "ape_get_status", "ape_status_string", "ape_decode_noalloc"]
 
 
 class ApeError(RuntimeError):
@@ -76,6 +76,9 @@ def load() -> C.CDLL:
                                         C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), vp]
         lib.ape_plan_last_launches.argtypes = [vp, C.POINTER(C.c_int32)]
         lib.ape_get_status.argtypes = [vp, C.POINTER(C.c_int32)]
+        lib.ape_decode_noalloc.argtypes = [C.POINTER(ape_shape_t), C.POINTER(ape_kv_pool_t), C.POINTER(ape_rows_t),
+                                           C.POINTER(ape_rows_t), vp, C.POINTER(ape_request_t), C.c_int32, C.c_float, C.c_float,
+                                           C.c_int64, C.c_int, vp, C.POINTER(C.c_int32)]
         lib.ape_status_string.argtypes = [C.c_int]
         lib.ape_status_string.restype = C.c_char_p
         for name in EXPORTS:
@@ -107,6 +110,36 @@ def _pool(k: torch.Tensor, v: torch.Tensor) -> ape_kv_pool_t:
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
     s = stream if stream is not None else torch.cuda.current_stream()
     return int(s.cuda_stream)
+
+
+def _request_array(requests: Sequence):
+    n = len(requests)
+    arr = (ape_request_t * max(n, 1))()
+    keep = []
+    for i, r in enumerate(requests):
+        spans = (ape_span_t * max(len(r.ctx), 1))(*[ape_span_t(int(s), int(l)) for s, l in r.ctx])
+        keep.append(spans)
+        arr[i] = ape_request_t(int(r.q_start), int(r.q_len), ape_span_t(*map(int, r.prefix)), spans, len(r.ctx),
+                               ape_span_t(*map(int, r.query_kv)), int(r.query_kv_capacity))
+    return arr, keep
+
+
+def decode_noalloc(*, H_q: int, H_kv: int, d: int, k_pool: torch.Tensor, v_pool: torch.Tensor, q: torch.Tensor,
+                   out: torch.Tensor, requests: Sequence, T: float, S: float, kv_extra: int = 0,
+                   lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0, device: int = 0,
+                   stream: Optional[torch.cuda.Stream] = None, want_status: bool = False) -> Optional[int]:
+    """ape_decode_noalloc: one decode step without a handle, a plan or a workspace; for callers that must not
+    allocate device memory.  The library keeps its scratch in a fixed 8 MiB device array; batches that do not fit
+    raise ApeError(APE_ERR_WORKSPACE).  With want_status the call synchronises and returns the device status word."""
+    shape = ape_shape_t(H_q, H_kv, d, softmax_scale)
+    pool, qr, orows = _pool(k_pool, v_pool), _rows(q), _rows(out)
+    arr, _keep = _request_array(requests)
+    st = C.c_int32(0)
+    _check(load().ape_decode_noalloc(C.byref(shape), C.byref(pool), C.byref(qr), C.byref(orows),
+                                     lse.data_ptr() if lse is not None else None, arr, len(requests), float(T), float(S),
+                                     int(kv_extra), int(device), _stream_ptr(stream), C.byref(st) if want_status else None),
+           "ape_decode_noalloc")
+    return int(st.value) if want_status else None
 
 
 class Handle:
