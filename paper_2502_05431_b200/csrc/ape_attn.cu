@@ -4,7 +4,7 @@
 // Every item is a run of 128-key tiles of ONE segment, so a plain online softmax per item is exact; the scaling
 // factor S of Eq. 5 acts on whole-segment log-sum-exps and is applied by the merge kernel afterwards.
 //
-// Roles (warp-specialised, 320 threads):
+// Roles (warp-specialised, 384 threads; warps 10-11 idle):
 //   warps 0-3 / 4-7  softmax of half 0 / half 1: one thread per row; S is read from TMEM, P = 2^(s - m) goes back
 //                    to TMEM as bf16 over the S columns, the running sum stays in a register; also the epilogue
 //   warp 8           producer: bulk tensor copies of Q, K and V tiles into 128-byte-swizzled shared memory
@@ -21,7 +21,9 @@ namespace {
 
 constexpr int kTileN = kAttnTileN;            // 128 keys per tile
 constexpr int kHalfRows = 128;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;               // three warpgroups; warps 10 and 11 only take part in the register hand-over
+constexpr int kRegsSoftmax = 216;            // registers per thread after the hand-over (two softmax warpgroups)
+constexpr int kRegsOther = 56;               // producer / MMA warpgroup
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr int kNK = 2;                        // K stages
@@ -68,8 +70,8 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t bar_k_full = bar0 + 16, bar_k_empty = bar_k_full + 8 * kNK;
     const uint32_t bar_v_full = bar_k_empty + 8 * kNK, bar_v_empty = bar_v_full + 8 * kNV;
     const uint32_t bar_s_full = bar_v_empty + 8 * kNV;         // [2]
-    const uint32_t bar_p_full = bar_s_full + 16;               // [2]
-    const uint32_t bar_o_full = bar_p_full + 16;               // [2]
+    const uint32_t bar_p_full = bar_s_full + 16;               // [2 halves][2 key halves]: P columns for keys 0-63 / 64-127 written
+    const uint32_t bar_o_full = bar_p_full + 32;               // [2]
     const uint32_t bar_done = bar_o_full + 16;
     __shared__ uint32_t tmem_base_smem;
     __shared__ int abort_flag;
@@ -83,7 +85,8 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int s = 0; s < kNV; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 1); }
         for (int w = 0; w < 2; ++w) {
             mbar_init(bar_s_full + 8 * w, 1);
-            mbar_init(bar_p_full + 8 * w, kHalfRows);
+            mbar_init(bar_p_full + 16 * w, 4);                 // one arrival per softmax warp
+            mbar_init(bar_p_full + 16 * w + 8, 4);
             mbar_init(bar_o_full + 8 * w, 1);
         }
         mbar_init(bar_done, 1);
@@ -112,8 +115,11 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         return g;
     };
 
+    // Register hand-over at the head of every role: the softmax threads hold a whole 128-column row of S in registers,
+    // the third warpgroup (producer, MMA issuer, two idle warps) gives its share up.
     if (warp == kProducerWarp) {
         // =============================== producer ====================================================================
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
         if (lane == 0) {
             tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
             uint32_t kcnt = 0, vcnt = 0, q_loads = 0;
@@ -137,8 +143,10 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                     ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
                 }
+                DevTile next_tile = p.tiles[item.tile_begin];
                 for (int t = item.tile_begin; t < item.tile_end; ++t) {
-                    const DevTile tile = p.tiles[t];
+                    const DevTile tile = next_tile;
+                    if (t + 1 < item.tile_end) next_tile = p.tiles[t + 1];
                     if (!tile_visible(tile, g)) continue;
                     {
                         const int s = kcnt % kNK; const uint32_t use = kcnt / kNK;
@@ -179,6 +187,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     } else if (warp == kMmaWarp) {
         // =============================== MMA issuer ==================================================================
         // All 32 lanes walk the loop and take part in the waits; lane 0 issues the tensor-core instructions.
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
         uint32_t kcnt = 0, vcnt = 0, q_loads = 0, pcnt = 0;
         int last_req = -1, last_head = -1, last_rb = -1;
         bool ok = true;
@@ -195,11 +204,13 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 mma_ss(tS[w], smem_desc_sw128(q_base + o, 16, 1024), smem_desc_sw128(k_base + o, 16, 1024), kIdescQK, ks > 0);
             }
         };
-        auto issue_pv = [&](int w, uint32_t v_base, bool accumulate) {
+        auto issue_pv = [&](int w, uint32_t v_base, bool accumulate, int key_half) {   // 4 k-steps: keys 64*key_half ..
             #pragma unroll
-            for (int ks = 0; ks < kTileN / 16; ++ks)
+            for (int k4 = 0; k4 < 4; ++k4) {
+                const int ks = key_half * 4 + k4;
                 mma_ts(tO[w], tS[w] + ks * 8, smem_desc_sw128(v_base + ks * 2048, kSlabBytes, 1024), kIdescPV,
                        (accumulate || ks > 0) ? 1u : 0u);
+            }
         };
         // V rows past the span may hold anything (even NaN bit patterns); P is 0 there, and 0 * NaN must stay 0.
         auto scrub_v = [&](uint8_t* v_tile, int n_valid) {
@@ -225,8 +236,10 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             bool have_prev = false, o_started = false;
             int prev_valid = kTileN;
             uint32_t prev_vs = 0, prev_vphase = 0;
+            DevTile next_tile = p.tiles[item.tile_begin];
             for (int t = item.tile_begin; t < item.tile_end; ++t) {
-                const DevTile tile = p.tiles[t];
+                const DevTile tile = next_tile;
+                if (t + 1 < item.tile_end) next_tile = p.tiles[t + 1];
                 if (!tile_visible(tile, g)) continue;
                 const int ksn = kcnt % kNK;
                 if (!wait_all(bar_k_full + 8 * ksn, (kcnt / kNK) & 1)) { ok = false; break; }
@@ -249,10 +262,14 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (prev_valid < kTileN) scrub_v(v_tile, prev_valid);
                     const uint32_t v_base = smem_u32(v_tile);
                     for (int w = 0; w < 2; ++w) {
-                        if (!wait_all(bar_p_full + 8 * w, pcnt & 1)) { ok = false; break; }
+                        if (!wait_all(bar_p_full + 16 * w, pcnt & 1)) { ok = false; break; }
+                        tc_fence_after();
+                        if (lane == 0) issue_pv(w, v_base, o_started, 0);
+                        __syncwarp();
+                        if (!wait_all(bar_p_full + 16 * w + 8, pcnt & 1)) { ok = false; break; }
                         tc_fence_after();
                         if (lane == 0) {
-                            issue_pv(w, v_base, o_started);
+                            issue_pv(w, v_base, o_started, 1);
                             if (w == 1) mma_commit(bar_v_empty + 8 * prev_vs);
                             issue_qk(w, k_base); mma_commit(bar_s_full + 8 * w);
                             if (w == 1) mma_commit(bar_k_empty + 8 * ksn);
@@ -271,10 +288,14 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (prev_valid < kTileN) scrub_v(v_tile, prev_valid);
                 const uint32_t v_base = smem_u32(v_tile);
                 for (int w = 0; w < 2; ++w) {
-                    if (!wait_all(bar_p_full + 8 * w, pcnt & 1)) { ok = false; break; }
+                    if (!wait_all(bar_p_full + 16 * w, pcnt & 1)) { ok = false; break; }
+                    tc_fence_after();
+                    if (lane == 0) issue_pv(w, v_base, o_started, 0);
+                    __syncwarp();
+                    if (!wait_all(bar_p_full + 16 * w + 8, pcnt & 1)) { ok = false; break; }
                     tc_fence_after();
                     if (lane == 0) {
-                        issue_pv(w, v_base, o_started);
+                        issue_pv(w, v_base, o_started, 1);
                         mma_commit(bar_o_full + 8 * w);
                         if (w == 1) mma_commit(bar_v_empty + 8 * prev_vs);
                     }
@@ -289,15 +310,16 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const long long t0 = clock64();
             while (!mbar_try_wait(bar_done, 0) && clock64() - t0 < (1ll << 24)) {}
         }
-    } else {
+    } else if (warp < 8) {
         // =============================== softmax + epilogue ==========================================================
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
         const int w = warp >> 2;
         const int r_local = (warp & 3) * 32 + lane;
         const int R = w * kHalfRows + r_local;                      // row inside the 256-row block
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + lane_base + (w ? kColS1 : kColS0);
         const uint32_t tO = tmem_base + lane_base + (w ? kColO1 : kColO0);
-        const uint32_t my_s_full = bar_s_full + 8 * w, my_p_full = bar_p_full + 8 * w, my_o_full = bar_o_full + 8 * w;
+        const uint32_t my_s_full = bar_s_full + 8 * w, my_p_full = bar_p_full + 16 * w, my_o_full = bar_o_full + 8 * w;
         uint32_t scnt = 0, ocnt = 0;
         bool ok = true;
 
@@ -313,8 +335,10 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             float m = -INFINITY, l = 0.f;
             int n_local = 0;
 
+            DevTile next_tile = p.tiles[item.tile_begin];
             for (int t = item.tile_begin; t < item.tile_end; ++t) {
-                const DevTile tile = p.tiles[t];
+                const DevTile tile = next_tile;
+                if (t + 1 < item.tile_end) next_tile = p.tiles[t + 1];      // in flight while this tile is processed
                 if (!tile_visible(tile, g)) continue;
                 if (!__all_sync(0xffffffffu, mbar_wait(my_s_full, scnt & 1, &abort_flag, p.status))) { ok = false; break; }
                 ++scnt;
@@ -379,11 +403,13 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         pk[i] = pack_bf16x2(p0, p1);
                     }
                     tmem_st32(tS + hh * 32, pk);
+                    // publish this half of P (64 keys): the PV product over it can start while the rest is computed
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(my_p_full + 8 * hh);
                 }
                 l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
-                tmem_st_wait();
-                tc_fence_before();
-                mbar_arrive(my_p_full);
                 ++n_local;
             }
             if (!ok) break;
@@ -437,6 +463,10 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (live) *reinterpret_cast<float2*>(p.ws_ml + row * 2) = make_float2(m, (n_local > 0) ? l : 0.f);
             }
         }
+    }
+
+    else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));     // warps 10, 11
     }
 
     // ---- teardown: every role has left its loop (normally or on an abort) ----------------------------------------------
