@@ -4,12 +4,12 @@
 // Every item is a run of 128-key tiles of ONE segment, so a plain online softmax per item is exact; the scaling
 // factor S of Eq. 5 acts on whole-segment log-sum-exps and is applied by the merge kernel afterwards.
 //
-// Roles (warp-specialised, 384 threads; warps 10-11 idle):
+// Roles (warp-specialised, 384 threads; warp 11 idle):
 //   warps 0-3 / 4-7  softmax of half 0 / half 1: one thread per row; S is read from TMEM, P = 2^(s - m) goes back
 //                    to TMEM as bf16 over the S columns, the running sum stays in a register; also the epilogue
 //   warp 8           producer: bulk tensor copies of Q, K and V tiles into 128-byte-swizzled shared memory
-//   warp 9           MMA issuer: S = Q K^T (both operands in shared memory) and O += P V (P from TMEM) with
-//                    tcgen05.mma, accumulators in TMEM; owns the TMEM allocation
+//   warps 9, 10      MMA issuers of half 0 / half 1: S = Q K^T (both operands in shared memory) and O += P V (P from
+//                    TMEM) with tcgen05.mma, accumulators in TMEM; warp 9 owns the TMEM allocation
 // The two halves run one tile apart, so that the tensor pipe works on one half while the other does its exponentials.
 #include "ape_common.cuh"
 #include "ape_kernels.h"
@@ -31,6 +31,31 @@ constexpr int kNV = 2;                        // V stages
 constexpr int kSlabBytes = 128 * 128;         // 128 rows x 64 bf16
 constexpr float kRescaleThreshold = 8.0f;     // base-2 units: O is rescaled only when the row maximum grew by more
 constexpr float kLn2 = 0.6931471805599453f;
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+// packed pairs of floats in one 64-bit register (fma.rn.f32x2 / add.rn.f32x2)
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
 
 struct ItemGeom {
     int rb;          // row block of this CTA for the item
@@ -70,9 +95,10 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t bar_k_full = bar0 + 16, bar_k_empty = bar_k_full + 8 * kNK;
     const uint32_t bar_v_full = bar_k_empty + 8 * kNK, bar_v_empty = bar_v_full + 8 * kNV;
     const uint32_t bar_s_full = bar_v_empty + 8 * kNV;         // [2]
-    const uint32_t bar_p_full = bar_s_full + 16;               // [2 halves][2 key halves]: P columns for keys 0-63 / 64-127 written
-    const uint32_t bar_o_full = bar_p_full + 32;               // [2]
+    const uint32_t bar_p_full = bar_s_full + 16;               // [2 halves][4 key quarters]: P columns of 32 keys written
+    const uint32_t bar_o_full = bar_p_full + 64;               // [2]
     const uint32_t bar_done = bar_o_full + 16;
+    const uint32_t bar_tok = bar_done + 8;                     // [2]: turn-taking of the two halves' exponential phases
     __shared__ uint32_t tmem_base_smem;
     __shared__ int abort_flag;
 
@@ -80,16 +106,16 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        mbar_init(bar_q_full, 1); mbar_init(bar_q_empty, 1);
-        for (int s = 0; s < kNK; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 1); }
-        for (int s = 0; s < kNV; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 1); }
+        mbar_init(bar_q_full, 1); mbar_init(bar_q_empty, 2);          // released by both MMA issuers
+        for (int s = 0; s < kNK; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 2); }
+        for (int s = 0; s < kNV; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 2); }
         for (int w = 0; w < 2; ++w) {
             mbar_init(bar_s_full + 8 * w, 1);
-            mbar_init(bar_p_full + 16 * w, 4);                 // one arrival per softmax warp
-            mbar_init(bar_p_full + 16 * w + 8, 4);
+            for (int qq = 0; qq < 4; ++qq) mbar_init(bar_p_full + 32 * w + 8 * qq, 4);   // one arrival per softmax warp
             mbar_init(bar_o_full + 8 * w, 1);
         }
-        mbar_init(bar_done, 1);
+        mbar_init(bar_done, 2);
+        mbar_init(bar_tok, 4); mbar_init(bar_tok + 8, 4);          // one arrival per softmax warp of the other half
         mbar_fence_init();
     }
     if (warp == kMmaWarp) {
@@ -116,7 +142,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     };
 
     // Register hand-over at the head of every role: the softmax threads hold a whole 128-column row of S in registers,
-    // the third warpgroup (producer, MMA issuer, two idle warps) gives its share up.
+    // the third warpgroup (producer, MMA issuers, one idle warp) gives its share up.
     if (warp == kProducerWarp) {
         // =============================== producer ====================================================================
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
@@ -184,35 +210,44 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 while (q_loads && !mbar_try_wait(bar_q_full, (q_loads - 1) & 1) && clock64() - t0 < (1ll << 24)) {}
             }
         }
-    } else if (warp == kMmaWarp) {
-        // =============================== MMA issuer ==================================================================
-        // All 32 lanes walk the loop and take part in the waits; lane 0 issues the tensor-core instructions.
+    } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
+        // =============================== MMA issuers: one warp per 128-row half =========================================
+        // Each half has its own issuing warp so that neither half ever queues behind the other's waits.  All 32 lanes
+        // walk the loop and take part in the waits; lane 0 issues the tensor-core instructions.
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+        const int w = warp - kMmaWarp;
         uint32_t kcnt = 0, vcnt = 0, q_loads = 0, pcnt = 0;
         int last_req = -1, last_head = -1, last_rb = -1;
         bool ok = true;
-        const uint32_t tS[2] = {tmem_base + kColS0, tmem_base + kColS1};
-        const uint32_t tO[2] = {tmem_base + kColO0, tmem_base + kColO1};
+        const uint32_t tS = tmem_base + (w ? kColS1 : kColS0);
+        const uint32_t tO = tmem_base + (w ? kColO1 : kColO0);
+        const uint32_t my_s_full = bar_s_full + 8 * w, my_p_full = bar_p_full + 32 * w, my_o_full = bar_o_full + 8 * w;
+        const uint32_t q_base = smem_u32(q_smem + w * kTileBytes);
         auto wait_all = [&](uint32_t bar, uint32_t parity) {
             return __all_sync(0xffffffffu, mbar_wait(bar, parity, &abort_flag, p.status)) != 0;
         };
-        auto issue_qk = [&](int w, uint32_t k_base) {
-            const uint32_t q_base = smem_u32(q_smem + w * kTileBytes);
+        // Descriptors differ from their tile's base descriptor only in the 14-bit start-address field (units of 16 B),
+        // so every MMA costs one add per operand instead of a descriptor build: the issuing lane shares its scheduler
+        // with two softmax warps and must stay lean.
+        const uint64_t q_desc0 = smem_desc_sw128(q_base, 16, 1024);
+        auto issue_qk = [&](uint32_t k_base) {
+            const uint64_t k_desc0 = smem_desc_sw128(k_base, 16, 1024);
             #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
-                const uint32_t o = (ks >> 2) * kSlabBytes + (ks & 3) * 32;
-                mma_ss(tS[w], smem_desc_sw128(q_base + o, 16, 1024), smem_desc_sw128(k_base + o, 16, 1024), kIdescQK, ks > 0);
+                const uint64_t o = static_cast<uint64_t>(((ks >> 2) * kSlabBytes + (ks & 3) * 32) >> 4);
+                mma_ss(tS, q_desc0 + o, k_desc0 + o, kIdescQK, ks > 0);
             }
         };
-        auto issue_pv = [&](int w, uint32_t v_base, bool accumulate, int key_half) {   // 4 k-steps: keys 64*key_half ..
+        auto issue_pv = [&](uint64_t v_desc0, bool accumulate, int key_quarter) {   // 2 k-steps: keys 32*key_quarter ..
             #pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4) {
-                const int ks = key_half * 4 + k4;
-                mma_ts(tO[w], tS[w] + ks * 8, smem_desc_sw128(v_base + ks * 2048, kSlabBytes, 1024), kIdescPV,
+            for (int k2 = 0; k2 < 2; ++k2) {
+                const int ks = key_quarter * 2 + k2;
+                mma_ts(tO, tS + ks * 8, v_desc0 + static_cast<uint64_t>((ks * 2048) >> 4), kIdescPV,
                        (accumulate || ks > 0) ? 1u : 0u);
             }
         };
         // V rows past the span may hold anything (even NaN bit patterns); P is 0 there, and 0 * NaN must stay 0.
+        // Both issuing warps clear the same rows with the same zeros before their own products: a benign overlap.
         auto scrub_v = [&](uint8_t* v_tile, int n_valid) {
             const int per_slab = (kTileN - n_valid) * 8;              // 16-byte chunks to clear in each slab
             for (int i = lane; i < per_slab * kSlabs; i += 32) {
@@ -222,6 +257,25 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             fence_proxy_async_smem();
             __syncwarp();
         };
+        // O += P V for the previous tile of this half, in two key halves as P is published
+        uint32_t prev_v_release = 0;
+        auto pv_prev = [&](uint32_t prev_vs, uint32_t prev_vphase, int prev_valid, bool o_started) {
+            if (!wait_all(bar_v_full + 8 * prev_vs, prev_vphase)) return false;
+            uint8_t* v_tile = v_smem + prev_vs * kTileBytes;
+            if (prev_valid < kTileN) scrub_v(v_tile, prev_valid);
+            const uint32_t v_base = smem_u32(v_tile);
+            const uint64_t v_desc0 = smem_desc_sw128(v_base, kSlabBytes, 1024);
+            #pragma unroll
+            for (int qq = 0; qq < 4; ++qq) {                      // P arrives in quarters of 32 keys
+                if (!wait_all(my_p_full + 8 * qq, pcnt & 1)) return false;
+                tc_fence_after();
+                if (lane == 0) issue_pv(v_desc0, o_started, qq);
+                __syncwarp();
+            }
+            prev_v_release = bar_v_empty + 8 * prev_vs;           // committed after the next S = Q K^T has been issued
+            ++pcnt;
+            return true;
+        };
 
         for (int it = item_begin; it < item_end && ok; ++it) {
             const DevItem item = p.items[it];
@@ -229,7 +283,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const DevReq rq = p.reqs[item.req];
             const ItemGeom g = geom(item, rq);
             if (!(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
-                if (q_loads > 0 && lane == 0) mma_commit(bar_q_empty);     // Q may be replaced once every MMA so far is done
+                if (q_loads > 0 && lane == 0) mma_commit(bar_q_empty);     // Q may be replaced once both halves' MMAs so far are done
                 if (!wait_all(bar_q_full, q_loads & 1)) { ok = false; break; }
                 ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
             }
@@ -247,61 +301,27 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ++kcnt;
                 const uint32_t vs = vcnt % kNV, vphase = (vcnt / kNV) & 1;
                 ++vcnt;
-                if (!have_prev) {
-                    tc_fence_after();
-                    if (lane == 0) {
-                        issue_qk(0, k_base); mma_commit(bar_s_full);
-                        issue_qk(1, k_base); mma_commit(bar_s_full + 8);
-                        mma_commit(bar_k_empty + 8 * ksn);
-                    }
-                    __syncwarp();
-                } else {
-                    // previous tile: O += P V, interleaved half by half with this tile's S = Q K^T
-                    if (!wait_all(bar_v_full + 8 * prev_vs, prev_vphase)) { ok = false; break; }
-                    uint8_t* v_tile = v_smem + prev_vs * kTileBytes;
-                    if (prev_valid < kTileN) scrub_v(v_tile, prev_valid);
-                    const uint32_t v_base = smem_u32(v_tile);
-                    for (int w = 0; w < 2; ++w) {
-                        if (!wait_all(bar_p_full + 16 * w, pcnt & 1)) { ok = false; break; }
-                        tc_fence_after();
-                        if (lane == 0) issue_pv(w, v_base, o_started, 0);
-                        __syncwarp();
-                        if (!wait_all(bar_p_full + 16 * w + 8, pcnt & 1)) { ok = false; break; }
-                        tc_fence_after();
-                        if (lane == 0) {
-                            issue_pv(w, v_base, o_started, 1);
-                            if (w == 1) mma_commit(bar_v_empty + 8 * prev_vs);
-                            issue_qk(w, k_base); mma_commit(bar_s_full + 8 * w);
-                            if (w == 1) mma_commit(bar_k_empty + 8 * ksn);
-                        }
-                        __syncwarp();
-                    }
-                    if (!ok) break;
-                    ++pcnt; o_started = true;
+                if (have_prev) {
+                    if (!pv_prev(prev_vs, prev_vphase, prev_valid, o_started)) { ok = false; break; }
+                    o_started = true;
                 }
+                tc_fence_after();
+                if (lane == 0) {
+                    issue_qk(k_base);
+                    mma_commit(my_s_full);                         // first: the softmax threads wait on this one
+                    mma_commit(bar_k_empty + 8 * ksn);
+                    if (prev_v_release) mma_commit(prev_v_release);
+                }
+                prev_v_release = 0;
+                __syncwarp();
                 have_prev = true; prev_valid = tile.n_valid; prev_vs = vs; prev_vphase = vphase;
             }
             if (ok && have_prev) {
                 // drain: the last tile's O += P V; o_full tells the softmax threads that O is final
-                if (!wait_all(bar_v_full + 8 * prev_vs, prev_vphase)) { ok = false; break; }
-                uint8_t* v_tile = v_smem + prev_vs * kTileBytes;
-                if (prev_valid < kTileN) scrub_v(v_tile, prev_valid);
-                const uint32_t v_base = smem_u32(v_tile);
-                for (int w = 0; w < 2; ++w) {
-                    if (!wait_all(bar_p_full + 16 * w, pcnt & 1)) { ok = false; break; }
-                    tc_fence_after();
-                    if (lane == 0) issue_pv(w, v_base, o_started, 0);
-                    __syncwarp();
-                    if (!wait_all(bar_p_full + 16 * w + 8, pcnt & 1)) { ok = false; break; }
-                    tc_fence_after();
-                    if (lane == 0) {
-                        issue_pv(w, v_base, o_started, 1);
-                        mma_commit(bar_o_full + 8 * w);
-                        if (w == 1) mma_commit(bar_v_empty + 8 * prev_vs);
-                    }
-                    __syncwarp();
-                }
-                ++pcnt;
+                if (!pv_prev(prev_vs, prev_vphase, prev_valid, o_started)) { ok = false; break; }
+                if (lane == 0) { mma_commit(my_o_full); mma_commit(prev_v_release); }
+                prev_v_release = 0;
+                __syncwarp();
             }
         }
         if (!ok) {
@@ -319,7 +339,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + lane_base + (w ? kColS1 : kColS0);
         const uint32_t tO = tmem_base + lane_base + (w ? kColO1 : kColO0);
-        const uint32_t my_s_full = bar_s_full + 8 * w, my_p_full = bar_p_full + 16 * w, my_o_full = bar_o_full + 8 * w;
+        const uint32_t my_s_full = bar_s_full + 8 * w, my_p_full = bar_p_full + 32 * w, my_o_full = bar_o_full + 8 * w;
         uint32_t scnt = 0, ocnt = 0;
         bool ok = true;
 
@@ -356,17 +376,18 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     #pragma unroll
                     for (int i = 0; i < kTileN; ++i) s[i] = (i < limit) ? s[i] : -INFINITY;
                 }
-                // eight independent running maxima keep the dependency chain short
+                // eight independent running maxima (3-input max) keep the dependency chain short
                 float mxa[8];
                 #pragma unroll
-                for (int k = 0; k < 8; ++k) mxa[k] = s[k];
+                for (int k = 0; k < 8; ++k) mxa[k] = max3(s[k], s[8 + k], s[16 + k]);
                 #pragma unroll
-                for (int i = 8; i < kTileN; i += 8) {
+                for (int i = 24; i < kTileN - 8; i += 16) {
                     #pragma unroll
-                    for (int k = 0; k < 8; ++k) mxa[k] = fmaxf(mxa[k], s[i + k]);
+                    for (int k = 0; k < 8; ++k) mxa[k] = max3(mxa[k], s[i + k], s[i + 8 + k]);
                 }
-                const float mx = fmaxf(fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])),
-                                       fmaxf(fmaxf(mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
+                #pragma unroll
+                for (int k = 0; k < 8; ++k) mxa[k] = fmaxf(mxa[k], s[kTileN - 8 + k]);
+                const float mx = fmaxf(max3(mxa[0], mxa[1], mxa[2]), fmaxf(max3(mxa[3], mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
                 const float m_new = fmaxf(m, mx * scale);
                 if (n_local == 0) {
                     m = m_new;
@@ -391,24 +412,46 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                 }
                 const float m_use = (m == -INFINITY) ? 0.f : m;
-                float sum[4] = {0.f, 0.f, 0.f, 0.f};
+                // The two halves take turns in the exponential phase: the special-function unit is the scarcest pipe, and
+                // alternating keeps one half in its exponentials while the other half's MMAs run.  Phase n of half 0 follows
+                // phase n-1 of half 1; phase n of half 1 follows phase n of half 0 (both halves see the same tiles).
+                {
+                    const uint32_t n = scnt - 1;
+                    bool turn = true;
+                    if (w == 0) { if (n > 0) turn = mbar_wait(bar_tok, (n - 1) & 1, &abort_flag, p.status); }
+                    else turn = mbar_wait(bar_tok + 8, n & 1, &abort_flag, p.status);
+                    if (!__all_sync(0xffffffffu, turn)) { ok = false; break; }
+                }
+                // p = 2^(s * scale - m): the multiply-subtract and the row sum run as packed two-float operations
+                const uint64_t scale2 = pack2(scale, scale), negm2 = pack2(-m_use, -m_use);
+                uint64_t sum2[2] = {0ull, 0ull};
+                // P is computed and published in quarters of 32 keys (16 packed registers): the PV product over a quarter
+                // runs while the next quarter's exponentials are computed, and only the last quarter's product plus the
+                // next S = Q K^T remain on this half's critical path.
                 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    uint32_t pk[32];
+                for (int qq = 0; qq < 4; ++qq) {
+                    uint32_t pk[16];
                     #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float p0 = fast_exp2(fmaf(s[hh * 64 + 2 * i], scale, -m_use));
-                        const float p1 = fast_exp2(fmaf(s[hh * 64 + 2 * i + 1], scale, -m_use));
-                        sum[i & 3] += p0 + p1;
+                    for (int i = 0; i < 16; ++i) {
+                        float x0, x1;
+                        unpack2(fma2(pack2(s[qq * 32 + 2 * i], s[qq * 32 + 2 * i + 1]), scale2, negm2), x0, x1);
+                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                        sum2[i & 1] = add2(sum2[i & 1], pack2(p0, p1));
                         pk[i] = pack_bf16x2(p0, p1);
                     }
-                    tmem_st32(tS + hh * 32, pk);
-                    // publish this half of P (64 keys): the PV product over it can start while the rest is computed
+                    if (qq == 3) {                                         // exponentials issued: the other half's turn
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_tok + 8 * (1 - w));
+                    }
+                    tmem_st16(tS + qq * 16, pk);
                     tmem_st_wait();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(my_p_full + 8 * hh);
+                    if (lane == 0) mbar_arrive(my_p_full + 8 * qq);
                 }
+                float sum[4];
+                unpack2(sum2[0], sum[0], sum[1]);
+                unpack2(sum2[1], sum[2], sum[3]);
                 l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
                 ++n_local;
             }
@@ -466,7 +509,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
 
     else {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));     // warps 10, 11
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));     // warp 11
     }
 
     // ---- teardown: every role has left its loop (normally or on an abort) ----------------------------------------------
