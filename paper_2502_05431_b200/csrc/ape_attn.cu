@@ -238,7 +238,8 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 mma_ss(tS, q_desc0 + o, k_desc0 + o, kIdescQK, ks > 0);
             }
         };
-        auto issue_pv = [&](uint64_t v_desc0, bool accumulate, int key_quarter) {   // 2 k-steps: keys 32*key_quarter ..
+        // P is zero past the last key that any row of the block may see, so the product stops there (rounded up to 16).
+        auto issue_pv = [&](uint64_t v_desc0, bool accumulate, int key_quarter) {   // keys 32*key_quarter .. +32
             #pragma unroll
             for (int k2 = 0; k2 < 2; ++k2) {
                 const int ks = key_quarter * 2 + k2;
@@ -246,31 +247,50 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                        (accumulate || ks > 0) ? 1u : 0u);
             }
         };
+        auto issue_pv_cut = [&](uint64_t v_desc0, bool accumulate, int key_quarter, int n16) {   // same, stopping at key n16
+            #pragma unroll
+            for (int k2 = 0; k2 < 2; ++k2) {
+                const int ks = key_quarter * 2 + k2;
+                if (ks * 16 < n16) mma_ts(tO, tS + ks * 8, v_desc0 + static_cast<uint64_t>((ks * 2048) >> 4), kIdescPV,
+                       (accumulate || ks > 0) ? 1u : 0u);
+            }
+        };
         // V rows past the span may hold anything (even NaN bit patterns); P is 0 there, and 0 * NaN must stay 0.
         // Both issuing warps clear the same rows with the same zeros before their own products: a benign overlap.
-        auto scrub_v = [&](uint8_t* v_tile, int n_valid) {
-            const int per_slab = (kTileN - n_valid) * 8;              // 16-byte chunks to clear in each slab
-            for (int i = lane; i < per_slab * kSlabs; i += 32) {
-                const int sl = i / per_slab, rem = i - sl * per_slab;
-                *reinterpret_cast<uint4*>(v_tile + sl * kSlabBytes + (n_valid + (rem >> 3)) * 128 + (rem & 7) * 16) = make_uint4(0, 0, 0, 0);
-            }
+        // Only rows that the product reads are cleared: [n_valid, n16).
+        auto scrub_v = [&](uint8_t* v_tile, int n_valid, int n16) {
+            const int per_slab = (n16 - n_valid) * 8;                 // 16-byte chunks to clear in each slab (fewer than 128)
+            #pragma unroll
+            for (int sl = 0; sl < kSlabs; ++sl)
+                for (int i = lane; i < per_slab; i += 32)
+                    *reinterpret_cast<uint4*>(v_tile + sl * kSlabBytes + (n_valid + (i >> 3)) * 128 + (i & 7) * 16) = make_uint4(0, 0, 0, 0);
             fence_proxy_async_smem();
             __syncwarp();
         };
         // O += P V for the previous tile of this half, in two key halves as P is published
         uint32_t prev_v_release = 0;
-        auto pv_prev = [&](uint32_t prev_vs, uint32_t prev_vphase, int prev_valid, bool o_started) {
+        auto pv_prev = [&](uint32_t prev_vs, uint32_t prev_vphase, int prev_valid, int prev_n16, bool o_started) {
             if (!wait_all(bar_v_full + 8 * prev_vs, prev_vphase)) return false;
             uint8_t* v_tile = v_smem + prev_vs * kTileBytes;
-            if (prev_valid < kTileN) scrub_v(v_tile, prev_valid);
+            if (prev_valid < prev_n16) scrub_v(v_tile, prev_valid, prev_n16);
             const uint32_t v_base = smem_u32(v_tile);
             const uint64_t v_desc0 = smem_desc_sw128(v_base, kSlabBytes, 1024);
-            #pragma unroll
-            for (int qq = 0; qq < 4; ++qq) {                      // P arrives in quarters of 32 keys
-                if (!wait_all(my_p_full + 8 * qq, pcnt & 1)) return false;
-                tc_fence_after();
-                if (lane == 0) issue_pv(v_desc0, o_started, qq);
-                __syncwarp();
+            if (prev_n16 == kTileN) {
+                #pragma unroll
+                for (int qq = 0; qq < 4; ++qq) {                  // P arrives in quarters of 32 keys
+                    if (!wait_all(my_p_full + 8 * qq, pcnt & 1)) return false;
+                    tc_fence_after();
+                    if (lane == 0) issue_pv(v_desc0, o_started, qq);
+                    __syncwarp();
+                }
+            } else {
+                #pragma unroll
+                for (int qq = 0; qq < 4; ++qq) {
+                    if (!wait_all(my_p_full + 8 * qq, pcnt & 1)) return false;
+                    tc_fence_after();
+                    if (lane == 0) issue_pv_cut(v_desc0, o_started, qq, prev_n16);
+                    __syncwarp();
+                }
             }
             prev_v_release = bar_v_empty + 8 * prev_vs;           // committed after the next S = Q K^T has been issued
             ++pcnt;
@@ -288,7 +308,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
             }
             bool have_prev = false, o_started = false;
-            int prev_valid = kTileN;
+            int prev_valid = kTileN, prev_n16 = kTileN;
             uint32_t prev_vs = 0, prev_vphase = 0;
             DevTile next_tile = p.tiles[item.tile_begin];
             for (int t = item.tile_begin; t < item.tile_end; ++t) {
@@ -302,7 +322,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const uint32_t vs = vcnt % kNV, vphase = (vcnt / kNV) & 1;
                 ++vcnt;
                 if (have_prev) {
-                    if (!pv_prev(prev_vs, prev_vphase, prev_valid, o_started)) { ok = false; break; }
+                    if (!pv_prev(prev_vs, prev_vphase, prev_valid, prev_n16, o_started)) { ok = false; break; }
                     o_started = true;
                 }
                 tc_fence_after();
@@ -314,11 +334,16 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 prev_v_release = 0;
                 __syncwarp();
-                have_prev = true; prev_valid = tile.n_valid; prev_vs = vs; prev_vphase = vphase;
+                {
+                    int n_keys = tile.n_valid;                     // keys any row of the block may see
+                    if (tile.flags & TILE_CAUSAL) n_keys = min(n_keys, g.last_tok + g.off - tile.key_base + 1);
+                    prev_n16 = (n_keys + 15) & ~15;
+                }
+                have_prev = true; prev_valid = min(tile.n_valid, prev_n16); prev_vs = vs; prev_vphase = vphase;
             }
             if (ok && have_prev) {
                 // drain: the last tile's O += P V; o_full tells the softmax threads that O is final
-                if (!pv_prev(prev_vs, prev_vphase, prev_valid, o_started)) { ok = false; break; }
+                if (!pv_prev(prev_vs, prev_vphase, prev_valid, prev_n16, o_started)) { ok = false; break; }
                 if (lane == 0) { mma_commit(my_o_full); mma_commit(prev_v_release); }
                 prev_v_release = 0;
                 __syncwarp();
