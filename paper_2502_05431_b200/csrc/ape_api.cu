@@ -357,13 +357,13 @@ int ape_attend_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
             assign_stream(runs, n_groups, p->n_sib, m);
             p->n_cta = n_groups * p->n_sib;
             p->n_slots = static_cast<int>(m.items.size()) * p->n_sib;
-            p->smem_bytes = attn_smem_bytes(D);
+            p->smem_bytes = attn_smem_bytes(D, 1);
             const size_t rows = static_cast<size_t>(p->n_slots) * kAttnRows;
             p->ws_bytes = ((rows * D * 4 + 255) & ~size_t(255)) + ((rows * 2 * 4 + 255) & ~size_t(255));
             rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
             if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
             if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
-            if (!rc && attn_set_smem_attr(D, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+            if (!rc && attn_set_smem_attr(D, 1, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
         }
         if (!rc) rc = upload(p, m);
     } catch (const std::bad_alloc&) {
@@ -434,11 +434,11 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
         for (auto& b : bins) { for (auto& it : b) m.items.push_back(it); m.cta_begin.push_back(static_cast<int32_t>(m.items.size())); }
         p->n_slots = 0;
         p->ws_bytes = 0;
-        p->smem_bytes = attn_smem_bytes(D);
+        p->smem_bytes = attn_smem_bytes(D, 2);
         rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
         if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
         if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
-        if (!rc && attn_set_smem_attr(D, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+        if (!rc && attn_set_smem_attr(D, 2, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
         if (!rc) rc = upload(p, m);
     } catch (const std::bad_alloc&) {
         rc = APE_ERR_NOMEM;
@@ -488,7 +488,7 @@ int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace
         ap.tiles = p->d_tiles; ap.items = p->d_items; ap.cta_item_begin = p->d_cta_begin; ap.reqs = p->d_reqs;
         ap.out = rows_desc(p->out); ap.lse_out = nullptr; ap.ws_o = ws_o; ap.ws_ml = ws_ml;
         ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c / T * kLog2e;
-        ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = p->n_sib; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
+        ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = p->n_sib; ap.n_q_bufs = 1; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
         if (launch_attn(D, p->tm_q, p->tm_k, p->tm_v, ap, p->n_cta, p->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
     }
     p->last_launches++;
@@ -514,7 +514,7 @@ int ape_encode_contexts(ape_plan_t p, void* workspace, size_t ws_bytes, void* st
     ap.tiles = p->d_tiles; ap.items = p->d_items; ap.cta_item_begin = p->d_cta_begin; ap.reqs = p->d_reqs;
     ap.out = rows_desc(p->out); ap.lse_out = p->lse; ap.ws_o = nullptr; ap.ws_ml = nullptr;
     ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c * kLog2e;
-    ap.G = p->G; ap.H_q = p->shape.n_q_heads; ap.n_sib = 1; ap.q_rows_are_pool = 1; ap.status = p->h->d_status;
+    ap.G = p->G; ap.H_q = p->shape.n_q_heads; ap.n_sib = 1; ap.n_q_bufs = 2; ap.q_rows_are_pool = 1; ap.status = p->h->d_status;
     if (launch_attn(p->shape.head_dim, p->tm_q, p->tm_k, p->tm_v, ap, p->n_cta, p->smem_bytes,
                     static_cast<cudaStream_t>(stream_v)) != cudaSuccess) return APE_ERR_CUDA;
     p->last_launches = 1;

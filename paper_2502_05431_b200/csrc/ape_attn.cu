@@ -4,7 +4,7 @@
 // Every item is a run of 128-key tiles of ONE segment, so a plain online softmax per item is exact; the scaling
 // factor S of Eq. 5 acts on whole-segment log-sum-exps and is applied by the merge kernel afterwards.
 //
-// Roles (warp-specialised, 384 threads; warp 11 idle):
+// Roles (warp-specialised, 384 threads; warp 11 loads Q in the double-buffered configuration, else idles):
 //   warps 0-3 / 4-7  softmax of half 0 / half 1: one thread per row; S is read from TMEM, P = 2^(s - m) goes back
 //                    to TMEM as bf16 over the S columns, the running sum stays in a register; also the epilogue
 //   warp 8           producer: bulk tensor copies of Q, K and V tiles into 128-byte-swizzled shared memory
@@ -27,7 +27,6 @@ constexpr int kRegsOther = 56;               // producer / MMA warpgroup
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr int kNK = 2;                        // K stages
-constexpr int kNV = 2;                        // V stages
 constexpr int kSlabBytes = 128 * 128;         // 128 rows x 64 bf16
 constexpr float kRescaleThreshold = 8.0f;     // base-2 units: O is rescaled only when the row maximum grew by more
 constexpr float kLn2 = 0.6931471805599453f;
@@ -71,13 +70,18 @@ __device__ __forceinline__ bool tile_visible(const DevTile& t, const ItemGeom& g
 
 }  // namespace
 
-template <int D>
+// QBUF: number of Q buffers.  Plans with long items (prefill) use one Q buffer and two stages each of K and V; plans
+// with many short items (encode) use two Q buffers, so that the next row block's Q arrives while the current one is
+// in use, and pay for them with a single V stage.
+template <int D, int QBUF>
 __global__ void __launch_bounds__(kThreads, 1)
 ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const AttnParams p)
 {
     constexpr int kSlabs = D / 64;
     constexpr int kTileBytes = kSlabs * kSlabBytes;            // one K or V tile, also one Q half
+    constexpr int kQBytes = 2 * kTileBytes;                    // both halves of a row block
+    constexpr int kNV = (QBUF == 2) ? 1 : 2;                   // V stages
     constexpr uint32_t kTmemCols = 512;
     constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 256 + D;
     constexpr uint32_t kIdescQK = idesc_bf16_f32(128, kTileN, 0, 0);
@@ -85,14 +89,14 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* q_smem = smem;                                    // 2 halves
-    uint8_t* k_smem = q_smem + 2 * kTileBytes;                 // kNK stages
+    uint8_t* q_smem = smem;                                    // QBUF buffers x 2 halves
+    uint8_t* k_smem = q_smem + QBUF * kQBytes;                 // kNK stages
     uint8_t* v_smem = k_smem + kNK * kTileBytes;               // kNV stages
     uint64_t* bars = reinterpret_cast<uint64_t*>(v_smem + kNV * kTileBytes);
     // barrier map
     const uint32_t bar0 = smem_u32(bars);
-    const uint32_t bar_q_full = bar0, bar_q_empty = bar0 + 8;
-    const uint32_t bar_k_full = bar0 + 16, bar_k_empty = bar_k_full + 8 * kNK;
+    const uint32_t bar_q_full = bar0, bar_q_empty = bar0 + 16;             // [QBUF] each
+    const uint32_t bar_k_full = bar0 + 32, bar_k_empty = bar_k_full + 8 * kNK;
     const uint32_t bar_v_full = bar_k_empty + 8 * kNK, bar_v_empty = bar_v_full + 8 * kNV;
     const uint32_t bar_s_full = bar_v_empty + 8 * kNV;         // [2]
     const uint32_t bar_p_full = bar_s_full + 16;               // [2 halves][4 key quarters]: P columns of 32 keys written
@@ -106,7 +110,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        mbar_init(bar_q_full, 1); mbar_init(bar_q_empty, 2);          // released by both MMA issuers
+        for (int b = 0; b < QBUF; ++b) { mbar_init(bar_q_full + 8 * b, 1); mbar_init(bar_q_empty + 8 * b, 2); }   // released by both MMA issuers
         for (int s = 0; s < kNK; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 2); }
         for (int s = 0; s < kNV; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 2); }
         for (int w = 0; w < 2; ++w) {
@@ -143,6 +147,22 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     // Register hand-over at the head of every role: the softmax threads hold a whole 128-column row of S in registers,
     // the third warpgroup (producer, MMA issuers, one idle warp) gives its share up.
+    // Q of one row block (both halves) into buffer n % QBUF, once the MMAs that read that buffer last are done.
+    auto load_q = [&](const DevItem& item, const DevReq& rq, const ItemGeom& g, uint32_t n) {
+        const uint32_t qb = n % QBUF, q_use = n / QBUF;
+        if (q_use > 0 && !mbar_wait(bar_q_empty + 8 * qb, (q_use - 1) & 1, &abort_flag, p.status)) return false;
+        mbar_expect_tx(bar_q_full + 8 * qb, kQBytes);
+        #pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            const int tok0 = rq.q_row0 + g.rb * TB + w * (kHalfRows / G);
+            #pragma unroll
+            for (int sl = 0; sl < kSlabs; ++sl)
+                tma_load_3d(smem_u32(q_smem + qb * kQBytes + w * kTileBytes + sl * kSlabBytes), &tm_q, bar_q_full + 8 * qb,
+                            sl * 64, item.kv_head * G, tok0);
+        }
+        return true;
+    };
+
     if (warp == kProducerWarp) {
         // =============================== producer ====================================================================
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
@@ -156,17 +176,8 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (sib >= item.n_sib) continue;
                 const DevReq rq = p.reqs[item.req];
                 const ItemGeom g = geom(item, rq);
-                if (!(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
-                    if (q_loads > 0 && !mbar_wait(bar_q_empty, (q_loads - 1) & 1, &abort_flag, p.status)) { ok = false; break; }
-                    mbar_expect_tx(bar_q_full, 2 * kTileBytes);
-                    #pragma unroll
-                    for (int w = 0; w < 2; ++w) {
-                        const int tok0 = rq.q_row0 + g.rb * TB + w * (kHalfRows / G);
-                        #pragma unroll
-                        for (int sl = 0; sl < kSlabs; ++sl)
-                            tma_load_3d(smem_u32(q_smem + w * kTileBytes + sl * kSlabBytes), &tm_q, bar_q_full,
-                                        sl * 64, item.kv_head * G, tok0);
-                    }
+                if (QBUF == 1 && !(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
+                    if (!load_q(item, rq, g, q_loads)) { ok = false; break; }
                     ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
                 }
                 DevTile next_tile = p.tiles[item.tile_begin];
@@ -207,7 +218,10 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     const uint32_t issued = (vcnt > static_cast<uint32_t>(s)) ? (vcnt - 1 - s) / kNV + 1 : 0;
                     while (issued && !mbar_try_wait(bar_v_full + 8 * s, (issued - 1) & 1) && clock64() - t0 < (1ll << 24)) {}
                 }
-                while (q_loads && !mbar_try_wait(bar_q_full, (q_loads - 1) & 1) && clock64() - t0 < (1ll << 24)) {}
+                for (uint32_t b = 0; b < QBUF; ++b) {
+                    const uint32_t issued = (q_loads > b) ? (q_loads - 1 - b) / QBUF + 1 : 0;
+                    while (QBUF == 1 && issued && !mbar_try_wait(bar_q_full + 8 * b, (issued - 1) & 1) && clock64() - t0 < (1ll << 24)) {}
+                }
             }
         }
     } else if (warp == kMmaWarp || warp == kMmaWarp + 1) {
@@ -222,14 +236,13 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t tS = tmem_base + (w ? kColS1 : kColS0);
         const uint32_t tO = tmem_base + (w ? kColO1 : kColO0);
         const uint32_t my_s_full = bar_s_full + 8 * w, my_p_full = bar_p_full + 32 * w, my_o_full = bar_o_full + 8 * w;
-        const uint32_t q_base = smem_u32(q_smem + w * kTileBytes);
         auto wait_all = [&](uint32_t bar, uint32_t parity) {
             return __all_sync(0xffffffffu, mbar_wait(bar, parity, &abort_flag, p.status)) != 0;
         };
         // Descriptors differ from their tile's base descriptor only in the 14-bit start-address field (units of 16 B),
         // so every MMA costs one add per operand instead of a descriptor build: the issuing lane shares its scheduler
         // with two softmax warps and must stay lean.
-        const uint64_t q_desc0 = smem_desc_sw128(q_base, 16, 1024);
+        uint64_t q_desc0 = smem_desc_sw128(smem_u32(q_smem + w * kTileBytes), 16, 1024);
         auto issue_qk = [&](uint32_t k_base) {
             const uint64_t k_desc0 = smem_desc_sw128(k_base, 16, 1024);
             #pragma unroll
@@ -292,7 +305,12 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     __syncwarp();
                 }
             }
-            prev_v_release = bar_v_empty + 8 * prev_vs;           // committed after the next S = Q K^T has been issued
+            if (kNV == 1) {                                       // single V stage: free it at once, the next V load is waiting
+                if (lane == 0) mma_commit(bar_v_empty + 8 * prev_vs);
+                __syncwarp();
+            } else {
+                prev_v_release = bar_v_empty + 8 * prev_vs;       // committed after the next S = Q K^T has been issued
+            }
             ++pcnt;
             return true;
         };
@@ -303,8 +321,11 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const DevReq rq = p.reqs[item.req];
             const ItemGeom g = geom(item, rq);
             if (!(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
-                if (q_loads > 0 && lane == 0) mma_commit(bar_q_empty);     // Q may be replaced once both halves' MMAs so far are done
-                if (!wait_all(bar_q_full, q_loads & 1)) { ok = false; break; }
+                // the Q buffer just used may be refilled once both halves' MMAs issued so far are done
+                if (q_loads > 0 && lane == 0) mma_commit(bar_q_empty + 8 * ((q_loads - 1) % QBUF));
+                const uint32_t qb = q_loads % QBUF;
+                if (!wait_all(bar_q_full + 8 * qb, (q_loads / QBUF) & 1)) { ok = false; break; }
+                if (QBUF > 1) q_desc0 = smem_desc_sw128(smem_u32(q_smem + qb * kQBytes + w * kTileBytes), 16, 1024);
                 ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
             }
             bool have_prev = false, o_started = false;
@@ -344,7 +365,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (ok && have_prev) {
                 // drain: the last tile's O += P V; o_full tells the softmax threads that O is final
                 if (!pv_prev(prev_vs, prev_vphase, prev_valid, prev_n16, o_started)) { ok = false; break; }
-                if (lane == 0) { mma_commit(my_o_full); mma_commit(prev_v_release); }
+                if (lane == 0) { mma_commit(my_o_full); if (prev_v_release) mma_commit(prev_v_release); }
                 prev_v_release = 0;
                 __syncwarp();
             }
@@ -534,7 +555,32 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
 
     else {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));     // warp 11
+        // =============================== warp 11: Q producer of the double-buffered configuration ==========================
+        // With two Q buffers the loads of Q run in their own thread, one row block ahead of the MMAs, instead of queueing
+        // behind the K/V loads of the current item.
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+        if (QBUF == 2 && lane == 0) {
+            tma_prefetch_desc(&tm_q);
+            uint32_t q_loads = 0;
+            int last_req = -1, last_head = -1, last_rb = -1;
+            bool ok = true;
+            for (int it = item_begin; it < item_end && ok; ++it) {
+                const DevItem item = p.items[it];
+                if (sib >= item.n_sib) continue;
+                const DevReq rq = p.reqs[item.req];
+                const ItemGeom g = geom(item, rq);
+                if (item.req == last_req && item.kv_head == last_head && g.rb == last_rb) continue;
+                if (!load_q(item, rq, g, q_loads)) { ok = false; break; }
+                ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
+            }
+            if (!ok) {
+                const long long t0 = clock64();
+                for (uint32_t b = 0; b < 2; ++b) {
+                    const uint32_t issued = (q_loads > b) ? (q_loads - 1 - b) / 2 + 1 : 0;
+                    while (issued && !mbar_try_wait(bar_q_full + 8 * b, (issued - 1) & 1) && clock64() - t0 < (1ll << 24)) {}
+                }
+            }
+        }
     }
 
     // ---- teardown: every role has left its loop (normally or on an abort) ----------------------------------------------
@@ -546,22 +592,27 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
 }
 
-size_t attn_smem_bytes(int D) {
+size_t attn_smem_bytes(int D, int q_bufs) {
     const size_t tile = static_cast<size_t>(D / 64) * kSlabBytes;
-    return 1024 + (2 + kNK + kNV) * tile + 256;
+    const int tiles = (q_bufs == 2) ? (4 + kNK + 1) : (2 + kNK + 2);     // Q halves + K stages + V stages
+    return 1024 + tiles * tile + 256;
 }
 
-cudaError_t attn_set_smem_attr(int D, size_t smem_bytes) {
-    if (D == 128)
-        return cudaFuncSetAttribute(ape_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes));
-    return cudaFuncSetAttribute(ape_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes));
+cudaError_t attn_set_smem_attr(int D, int q_bufs, size_t smem_bytes) {
+    const int n = static_cast<int>(smem_bytes);
+    if (D == 128 && q_bufs == 2) return cudaFuncSetAttribute(ape_attn_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (D == 128) return cudaFuncSetAttribute(ape_attn_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (q_bufs == 2) return cudaFuncSetAttribute(ape_attn_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    return cudaFuncSetAttribute(ape_attn_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
 }
 
 cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                         const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream)
 {
-    if (D == 128) ape_attn_kernel<128><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
-    else ape_attn_kernel<64><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
+    if (D == 128 && p.n_q_bufs == 2) ape_attn_kernel<128, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
+    else if (D == 128) ape_attn_kernel<128, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
+    else if (p.n_q_bufs == 2) ape_attn_kernel<64, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
+    else ape_attn_kernel<64, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
     return cudaGetLastError();
 }
 

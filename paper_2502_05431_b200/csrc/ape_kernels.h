@@ -46,12 +46,13 @@ struct AttnParams {
     int32_t G;
     int32_t H_q;
     int32_t n_sib;                   // sibling CTAs per group (row blocks that stream the same tiles together)
+    int32_t n_q_bufs;                // 1: long items (prefill); 2: many short items (encode), see the kernel
     int32_t q_rows_are_pool;         // encode: Q / O rows are pool tokens (row = context start + i)
     int* status;
 };
 
-size_t attn_smem_bytes(int D);
-cudaError_t attn_set_smem_attr(int D, size_t smem_bytes);
+size_t attn_smem_bytes(int D, int q_bufs);
+cudaError_t attn_set_smem_attr(int D, int q_bufs, size_t smem_bytes);
 cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                         const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream);
 
