@@ -281,7 +281,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             __syncwarp();
         };
         // O += P V for the previous tile of this half, in two key halves as P is published
-        uint32_t prev_v_release = 0;
+        uint32_t prev_v_release = 0, pending_q_release = 0;
         auto pv_prev = [&](uint32_t prev_vs, uint32_t prev_vphase, int prev_valid, int prev_n16, bool o_started) {
             if (!wait_all(bar_v_full + 8 * prev_vs, prev_vphase)) return false;
             uint8_t* v_tile = v_smem + prev_vs * kTileBytes;
@@ -321,8 +321,14 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const DevReq rq = p.reqs[item.req];
             const ItemGeom g = geom(item, rq);
             if (!(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
-                // the Q buffer just used may be refilled once both halves' MMAs issued so far are done
-                if (q_loads > 0 && lane == 0) mma_commit(bar_q_empty + 8 * ((q_loads - 1) % QBUF));
+                // The Q buffer just used may be refilled once both halves' MMAs issued so far are done.  A commit that
+                // follows another commit holds the issuing thread until the tensor pipe has drained, so with two Q
+                // buffers this one is put off until the next S = Q K^T is on its way (with one buffer that product waits
+                // for the refill, so the commit cannot wait for it).
+                if (q_loads > 0) {
+                    if (QBUF == 1) { if (lane == 0) mma_commit(bar_q_empty); }
+                    else pending_q_release = bar_q_empty + 8 * ((q_loads - 1) % QBUF);
+                }
                 const uint32_t qb = q_loads % QBUF;
                 if (!wait_all(bar_q_full + 8 * qb, (q_loads / QBUF) & 1)) { ok = false; break; }
                 if (QBUF > 1) q_desc0 = smem_desc_sw128(smem_u32(q_smem + qb * kQBytes + w * kTileBytes), 16, 1024);
@@ -352,8 +358,9 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     mma_commit(my_s_full);                         // first: the softmax threads wait on this one
                     mma_commit(bar_k_empty + 8 * ksn);
                     if (prev_v_release) mma_commit(prev_v_release);
+                    if (pending_q_release) mma_commit(pending_q_release);
                 }
-                prev_v_release = 0;
+                prev_v_release = 0; pending_q_release = 0;
                 __syncwarp();
                 {
                     int n_keys = tile.n_valid;                     // keys any row of the block may see
@@ -365,8 +372,9 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (ok && have_prev) {
                 // drain: the last tile's O += P V; o_full tells the softmax threads that O is final
                 if (!pv_prev(prev_vs, prev_vphase, prev_valid, prev_n16, o_started)) { ok = false; break; }
-                if (lane == 0) { mma_commit(my_o_full); if (prev_v_release) mma_commit(prev_v_release); }
-                prev_v_release = 0;
+                // o_full only: the stage release waits for the next item's first product (nobody needs it sooner than that,
+                // and after the last item nobody needs it at all)
+                if (lane == 0) mma_commit(my_o_full);
                 __syncwarp();
             }
         }
@@ -514,20 +522,24 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const int h = item.kv_head * G + hg;
                 __nv_bfloat16* dst = p.out.data + static_cast<int64_t>(rq.q_row0 + tok) * p.out.token_stride
                                      + static_cast<int64_t>(h) * p.out.head_stride;
+                const bool wide_ok = (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;
                 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t o[32];
                     tmem_ld32(tO + c * 32, o);
                     tmem_ld_wait();
                     if (live) {
+                        uint32_t pk[16];
                         #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            uint4 v;
-                            v.x = pack_bf16x2(__uint_as_float(o[8 * i + 0]) * inv, __uint_as_float(o[8 * i + 1]) * inv);
-                            v.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv, __uint_as_float(o[8 * i + 3]) * inv);
-                            v.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv, __uint_as_float(o[8 * i + 5]) * inv);
-                            v.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv, __uint_as_float(o[8 * i + 7]) * inv);
-                            *reinterpret_cast<uint4*>(dst + c * 32 + i * 8) = v;
+                        for (int i = 0; i < 16; ++i)
+                            pk[i] = pack_bf16x2(__uint_as_float(o[2 * i]) * inv, __uint_as_float(o[2 * i + 1]) * inv);
+                        if (wide_ok) {                 // 32-byte stores: one full sector per instruction
+                            st_global_v8(dst + c * 32, pk[0], pk[1], pk[2], pk[3], pk[4], pk[5], pk[6], pk[7]);
+                            st_global_v8(dst + c * 32 + 16, pk[8], pk[9], pk[10], pk[11], pk[12], pk[13], pk[14], pk[15]);
+                        } else {
+                            #pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                *reinterpret_cast<uint4*>(dst + c * 32 + i * 8) = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
                         }
                     }
                 }
@@ -542,10 +554,11 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         uint32_t o[32];
                         tmem_ld32(tO + c * 32, o);
                         tmem_ld_wait();
-                        if (live) {
+                        if (live) {                        // workspace rows are 256-byte aligned
                             #pragma unroll
-                            for (int i = 0; i < 8; ++i)
-                                *reinterpret_cast<uint4*>(dst + c * 32 + i * 4) = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+                            for (int i = 0; i < 4; ++i)
+                                st_global_v8(dst + c * 32 + i * 8, o[8 * i], o[8 * i + 1], o[8 * i + 2], o[8 * i + 3],
+                                             o[8 * i + 4], o[8 * i + 5], o[8 * i + 6], o[8 * i + 7]);
                         }
                     }
                 }
