@@ -179,6 +179,16 @@ void assign_stream(const std::vector<Run>& runs, int n_bins, int slot_mult, Host
     while (static_cast<int>(m.cta_begin.size()) < n_bins + 1) m.cta_begin.push_back(static_cast<int32_t>(m.items.size()));
 }
 
+// Every item carries a copy of its request's geometry and of its first tile record.
+void finish_items(HostMeta& m) {
+    for (auto& it : m.items) {
+        const DevReq& rq = m.reqs[it.req];
+        it.q_row0 = rq.q_row0; it.q_len = rq.q_len; it.l_k = rq.l_k; it.pad = 0;
+        if (it.tile_begin < static_cast<int32_t>(m.tiles.size())) it.first_tile = m.tiles[it.tile_begin];
+        else it.first_tile = DevTile{0, 0, 0, 0};
+    }
+}
+
 int upload(ape_plan_t p, const HostMeta& m) {
     auto rnd = [](size_t x) { return (x + 255) & ~size_t(255); };
     const size_t b_tiles = rnd(m.tiles.size() * sizeof(DevTile) + 16), b_items = rnd(m.items.size() * sizeof(DevItem) + 16),
@@ -365,7 +375,7 @@ int ape_attend_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
             if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
             if (!rc && attn_set_smem_attr(D, 1, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
         }
-        if (!rc) rc = upload(p, m);
+        if (!rc) { finish_items(m); rc = upload(p, m); }
     } catch (const std::bad_alloc&) {
         rc = APE_ERR_NOMEM;
     }
@@ -417,7 +427,9 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
                 for (int rb = 0; rb < RB; ++rb) {
                     const int64_t last_tok = std::min<int64_t>(ctx[i].len, static_cast<int64_t>(rb + 1) * TB) - 1;
                     const int vis = n_pref + static_cast<int>(last_tok / tile) + 1;     // tiles this row block can see
-                    DevItem it{i, hh, rb, t0, std::min(t1, t0 + vis), 0, SEG_FINAL, 1};
+                    DevItem it{};
+                    it.req = i; it.kv_head = hh; it.row_block = rb; it.tile_begin = t0; it.tile_end = std::min(t1, t0 + vis);
+                    it.slot = 0; it.seg = SEG_FINAL; it.n_sib = 1;
                     work.push_back(Work{it, vis});
                 }
         }
@@ -439,7 +451,7 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
         if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
         if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
         if (!rc && attn_set_smem_attr(D, 2, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
-        if (!rc) rc = upload(p, m);
+        if (!rc) { finish_items(m); rc = upload(p, m); }
     } catch (const std::bad_alloc&) {
         rc = APE_ERR_NOMEM;
     }
@@ -679,6 +691,7 @@ int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, cons
             }
         }
         assign_stream(runs, n_cta, 1, m);
+        finish_items(m);
         auto rnd = [](size_t x) { return (x + 255) & ~size_t(255); };
         o_tiles = 256;                                                     // after the status word
         o_items = o_tiles + rnd(m.tiles.size() * sizeof(DevTile));

@@ -56,6 +56,10 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     return r;
 }
 
+__device__ __forceinline__ void prefetch_l1(const void* ptr) {
+    asm volatile("prefetch.global.L1 [%0];" ::"l"(ptr));
+}
+
 struct ItemGeom {
     int rb;          // row block of this CTA for the item
     int last_tok;    // last live query token of the row block
@@ -173,14 +177,15 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             bool ok = true;
             for (int it = item_begin; it < item_end && ok; ++it) {
                 const DevItem item = p.items[it];
+                if (it + 1 < item_end) prefetch_l1(&p.items[it + 1]);   // the next item's record is in cache when its turn comes
                 if (sib >= item.n_sib) continue;
-                const DevReq rq = p.reqs[item.req];
+                const DevReq rq{item.q_row0, item.q_len, item.l_k, 0};
                 const ItemGeom g = geom(item, rq);
                 if (QBUF == 1 && !(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
                     if (!load_q(item, rq, g, q_loads)) { ok = false; break; }
                     ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
                 }
-                DevTile next_tile = p.tiles[item.tile_begin];
+                DevTile next_tile = item.first_tile;
                 for (int t = item.tile_begin; t < item.tile_end; ++t) {
                     const DevTile tile = next_tile;
                     if (t + 1 < item.tile_end) next_tile = p.tiles[t + 1];
@@ -317,8 +322,9 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
         for (int it = item_begin; it < item_end && ok; ++it) {
             const DevItem item = p.items[it];
+            if (it + 1 < item_end) prefetch_l1(&p.items[it + 1]);       // the next item's record is in cache when its turn comes
             if (sib >= item.n_sib) continue;
-            const DevReq rq = p.reqs[item.req];
+            const DevReq rq{item.q_row0, item.q_len, item.l_k, 0};
             const ItemGeom g = geom(item, rq);
             if (!(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
                 // The Q buffer just used may be refilled once both halves' MMAs issued so far are done.  A commit that
@@ -337,7 +343,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             bool have_prev = false, o_started = false;
             int prev_valid = kTileN, prev_n16 = kTileN;
             uint32_t prev_vs = 0, prev_vphase = 0;
-            DevTile next_tile = p.tiles[item.tile_begin];
+            DevTile next_tile = item.first_tile;
             for (int t = item.tile_begin; t < item.tile_end; ++t) {
                 const DevTile tile = next_tile;
                 if (t + 1 < item.tile_end) next_tile = p.tiles[t + 1];
@@ -399,8 +405,9 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
         for (int it = item_begin; it < item_end && ok; ++it) {
             const DevItem item = p.items[it];
+            if (it + 1 < item_end) prefetch_l1(&p.items[it + 1]);       // the next item's record is in cache when its turn comes
             if (sib >= item.n_sib) continue;
-            const DevReq rq = p.reqs[item.req];
+            const DevReq rq{item.q_row0, item.q_len, item.l_k, 0};
             const ItemGeom g = geom(item, rq);
             const int tok = g.rb * TB + R / G;
             const int hg = R % G;
@@ -409,7 +416,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             float m = -INFINITY, l = 0.f;
             int n_local = 0;
 
-            DevTile next_tile = p.tiles[item.tile_begin];
+            DevTile next_tile = item.first_tile;
             for (int t = item.tile_begin; t < item.tile_end; ++t) {
                 const DevTile tile = next_tile;
                 if (t + 1 < item.tile_end) next_tile = p.tiles[t + 1];      // in flight while this tile is processed
@@ -579,8 +586,9 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             bool ok = true;
             for (int it = item_begin; it < item_end && ok; ++it) {
                 const DevItem item = p.items[it];
+                if (it + 1 < item_end) prefetch_l1(&p.items[it + 1]);   // the next item's record is in cache when its turn comes
                 if (sib >= item.n_sib) continue;
-                const DevReq rq = p.reqs[item.req];
+                const DevReq rq{item.q_row0, item.q_len, item.l_k, 0};
                 const ItemGeom g = geom(item, rq);
                 if (item.req == last_req && item.kv_head == last_head && g.rb == last_rb) continue;
                 if (!load_q(item, rq, g, q_loads)) { ok = false; break; }

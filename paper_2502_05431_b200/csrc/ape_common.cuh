@@ -30,7 +30,15 @@ struct DevItem {
     int32_t slot;        // partial slot of sibling 0; sibling s writes slot + s
     int32_t seg;         // SEG_OTHER (prefix + query segment), SEG_CTX, or SEG_FINAL (encode: write O directly)
     int32_t n_sib;       // live siblings of this item (row blocks that exist)
+    // copies of the request geometry and of the first tile record, so that an item is ONE 64-byte load that the
+    // tensor-core kernel fetches an item ahead (no dependent loads when it moves to the next item)
+    int32_t q_row0;      // first row of Q / O of the request (encode: context start)
+    int32_t q_len;       // query rows of the request
+    int32_t l_k;         // keys in the query segment at planning time (encode: context length)
+    int32_t pad;
+    DevTile first_tile;  // tiles[tile_begin]
 };
+static_assert(sizeof(DevItem) == 64, "DevItem is one 64-byte record");
 enum : int32_t { SEG_OTHER = 0, SEG_CTX = 1, SEG_FINAL = 2 };
 
 // Per request (attend) / per context (encode) row geometry.
