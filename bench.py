@@ -50,6 +50,28 @@ def decode_bytes(n_req: int, tokens_per_req: int) -> float:
     return n_req * (tokens_per_req * 4.0 * H_KV * D + 2 * 2.0 * H_Q * D)
 
 
+# DRAM traffic per full-size launch (dram__bytes_read.sum + dram__bytes_write.sum), taken from the ncu captures
+# summarised under profiles/ on smaller cases and scaled by the units processed (traffic grows in proportion to the
+# cached tokens).  Valid only for the kernel sources the counters were taken with: the figure is dropped (null) as
+# soon as the hash of those sources changes.
+NCU_TRAFFIC = {
+    "prefill": {"bytes": 2 * (267.07e6 + 10.48e6), "sources": ["ape_attn.cu", "ape_tcgen05.cuh", "ape_common.cuh"], "sha": "dc520fcc2a4e5e36"},
+    "decode": {"bytes": (1.05515e9 + 4.08e6) * (8409907200.0 / 1053835264.0), "sources": ["ape_decode.cu", "ape_common.cuh"], "sha": "40414ccd4470df96"},
+}
+
+
+def ncu_traffic(which: str):
+    import hashlib
+    t = NCU_TRAFFIC[which]
+    h = hashlib.sha256()
+    try:
+        for f in t["sources"]:
+            h.update(open(os.path.join(ROOT, "paper_2502_05431_b200", "csrc", f), "rb").read())
+    except OSError:
+        return None
+    return t["bytes"] if h.hexdigest()[:16] == t["sha"] else None
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -161,7 +183,7 @@ def main():
     if args.impl == "reference":
         return run_reference(args)
 
-    from paper_2502_05431_b200 import libape, workloads as wl
+    from paper_2502_05431_b200 import dist_util, libape, workloads as wl
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -175,7 +197,7 @@ def main():
 
     libape.load()                                  # fails loudly if the CUDA library is missing
     h = libape.Handle(local_rank)
-    seed = 100 * rank                              # every rank works on its own replica (weak scaling, no exchange)
+    seed = dist_util.replica_seed(0, rank)         # every rank works on its own replica (weak scaling, no exchange)
 
     # ---- inputs, resident in HBM ------------------------------------------------------------------------------------
     pb = wl.config4(seed=seed, with_encode_q=True, device=str(dev))          # prefill + encode share this pool
@@ -233,10 +255,7 @@ def main():
     t_pre = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
     t_dec = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
     t_step = events[0][0].elapsed_time(events[-1][3]) / args.steps
-    times = torch.tensor([t_enc, t_pre, t_dec, t_step], dtype=torch.float64, device=dev)
-    if dist:
-        td.all_reduce(times, op=td.ReduceOp.MAX)
-    t_enc, t_pre, t_dec, t_step = times.tolist()
+    t_enc, t_pre, t_dec, t_step = dist_util.max_over_ranks([t_enc, t_pre, t_dec, t_step], dev)
 
     # ---- end to end through the host-buffer entry point (prefill half of the metric) ---------------------------------
     e2e = None
@@ -250,11 +269,9 @@ def main():
             h2d, d2h = plan_p.attend_host(pb.T, pb.S, ws_p, hq, hk, hv, hout)
         torch.cuda.synchronize()
         dt = (time.time() - t0) / max(args.e2e_steps, 1)
-        tdt = torch.tensor([dt], dtype=torch.float64, device=dev)
-        if dist:
-            td.all_reduce(tdt, op=td.ReduceOp.MAX)
-        e2e = {"value": world * fl_prefill / tdt.item() / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "ms_per_step": 1e3 * tdt.item(), "what": "ape_attend_host: Q + K/V pools host->device, attend, O device->host"}
+        dt = dist_util.max_over_ranks([dt], dev)[0]
+        e2e = {"value": dist_util.whole_job_rate(fl_prefill, world, dt * 1e3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": 1e3 * dt, "what": "ape_attend_host: Q + K/V pools host->device, attend, O device->host"}
 
     if rank != 0:
         if dist:
@@ -267,10 +284,11 @@ def main():
     gbs_decode = by_decode / (t_dec * 1e-3) / 1e9
     # the prefill kernel runs alone for ~0.5 ms inside a multi-ms step: sustained peak is the fair denominator
     roof = {"bound": "tensor", "kernel": "ape_attn_kernel<128> (+ merge) on the 128K prefill", "achieved": tf_prefill,
-            "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "frac": tf_prefill / peaks["tf_sustained"], "traffic": None,
+            "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "frac": tf_prefill / peaks["tf_sustained"], "traffic": ncu_traffic("prefill"),
+            "algorithmic_bytes": (L_P + N_CTX * L_CTX + L_Q) * 4.0 * H_KV * D + 2 * 2.0 * L_Q * H_Q * D,
             "peak_source": f"{peaks['source']} bf16 sustained", "frac_of_nominal_2250": tf_prefill / 2250.0}
     roof_dec = {"bound": "hbm", "kernel": "ape_decode_kernel<128> (+ merge)", "achieved": gbs_decode, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": gbs_decode / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peaks['source']} copy",
+                "unit": "GB/s", "frac": gbs_decode / peaks["hbm_gbs"], "traffic": ncu_traffic("decode"), "peak_source": f"{peaks['source']} copy",
                 "frac_of_nominal_8000": gbs_decode / 8000.0}
     cpu = None if args.no_cpu_baseline else cpu_oracle_sample()
     line = {
