@@ -55,7 +55,7 @@ def decode_bytes(n_req: int, tokens_per_req: int) -> float:
 # cached tokens).  Valid only for the kernel sources the counters were taken with: the figure is dropped (null) as
 # soon as the hash of those sources changes.
 NCU_TRAFFIC = {
-    "prefill": {"bytes": 2 * (267.07e6 + 10.48e6), "sources": ["ape_attn.cu", "ape_tcgen05.cuh", "ape_common.cuh"], "sha": "dc520fcc2a4e5e36"},
+    "prefill": {"bytes": 2 * (267.07e6 + 10.48e6), "sources": ["ape_attn.cu", "ape_tcgen05.cuh", "ape_common.cuh"], "sha": "9d2800857a8865cb"},
     "decode": {"bytes": (1.05515e9 + 4.08e6) * (8409907200.0 / 1053835264.0), "sources": ["ape_decode.cu", "ape_common.cuh"], "sha": "40414ccd4470df96"},
 }
 

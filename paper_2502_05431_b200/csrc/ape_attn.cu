@@ -619,8 +619,27 @@ size_t attn_smem_bytes(int D, int q_bufs) {
     return 1024 + tiles * tile + 256;
 }
 
+// The register hand-over only works if the registers that the third warpgroup gives up cover what the two softmax
+// warpgroups ask for: setmaxnreg.inc waits, without a bound, until they are there.  The launch-time register count is
+// the compiler's choice, so it is checked here, on the host, before the kernel is ever launched.
+template <typename K>
+static cudaError_t check_register_handover(K kernel) {
+    cudaFuncAttributes attr;
+    const cudaError_t e = cudaFuncGetAttributes(&attr, kernel);
+    if (e != cudaSuccess) return e;
+    const int freed = (attr.numRegs - kRegsOther) * 128;
+    const int wanted = (kRegsSoftmax - attr.numRegs) * 256;
+    return (attr.numRegs >= kRegsOther && attr.numRegs <= kRegsSoftmax && freed >= wanted) ? cudaSuccess : cudaErrorLaunchOutOfResources;
+}
+
 cudaError_t attn_set_smem_attr(int D, int q_bufs, size_t smem_bytes) {
     const int n = static_cast<int>(smem_bytes);
+    cudaError_t e;
+    if (D == 128 && q_bufs == 2) e = check_register_handover(ape_attn_kernel<128, 2>);
+    else if (D == 128) e = check_register_handover(ape_attn_kernel<128, 1>);
+    else if (q_bufs == 2) e = check_register_handover(ape_attn_kernel<64, 2>);
+    else e = check_register_handover(ape_attn_kernel<64, 1>);
+    if (e != cudaSuccess) return e;
     if (D == 128 && q_bufs == 2) return cudaFuncSetAttribute(ape_attn_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
     if (D == 128) return cudaFuncSetAttribute(ape_attn_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
     if (q_bufs == 2) return cudaFuncSetAttribute(ape_attn_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);

@@ -34,6 +34,8 @@ def _check_batch(b, mode, rows=None, lse_tol=2e-3, **kw):
     dict(**LLAMA, l_P=0, ctx_lens=[[333]], l_k=1, T=0.5, S=1.2, shuffle_ctx=True),
     dict(H_q=16, H_kv=1, d=128, l_P=64, ctx_lens=[[256] * 3], l_k=65, T=0.9, S=0.9),                # G = 16
     dict(H_q=8, H_kv=8, d=64, l_P=3, ctx_lens=[[100, 100]], l_k=9, T=0.9, S=0.5),                   # G = 1
+    dict(H_q=16, H_kv=8, d=128, l_P=9, ctx_lens=[[65, 190]], l_k=2, T=0.9, S=0.9),                  # G = 2
+    dict(H_q=8, H_kv=1, d=64, l_P=70, ctx_lens=[[64] * 5], l_k=130, T=1.3, S=0.9),                  # G = 8, d = 64
 ])
 def test_decode_small(kw):
     b = wl.make_batch(l_q=1, seed=1, name="decode_small", **kw)
@@ -90,6 +92,9 @@ def test_prefill_config1_tiny():
     dict(H_q=8, H_kv=8, d=64, l_P=10, ctx_lens=[[300]], l_q=300, T=0.8, S=1.1),             # G = 1, d = 64, 2 row blocks
     dict(H_q=16, H_kv=1, d=128, l_P=64, ctx_lens=[[256] * 4], l_q=40, T=0.9, S=0.9),        # G = 16
     dict(**LLAMA, l_P=64, ctx_lens=[[512] * 9], l_q=320, T=0.9, S=0.9),                     # 5 row blocks > 4 siblings
+    dict(H_q=16, H_kv=8, d=128, l_P=40, ctx_lens=[[300], [10, 500]], l_q=130, T=0.9, S=0.9),   # G = 2, 2 requests
+    dict(H_q=8, H_kv=1, d=64, l_P=1, ctx_lens=[[129]], l_q=33, l_k=40, T=0.7, S=1.0),            # G = 8, d = 64
+    dict(**LLAMA, l_P=0, ctx_lens=[[4096]], l_q=1, l_k=1, T=0.9, S=0.9),                         # a single query row
 ])
 def test_prefill_shapes(kw):
     b = wl.make_batch(seed=4, name="prefill", **kw)
@@ -175,7 +180,27 @@ def _check_encode(b):
     dict(**LLAMA, l_P=32, ctx_lens=[[256] * 10]),                                  # config 2
     dict(**LLAMA, l_P=0, ctx_lens=[[1, 129, 0, 300]], gap=3),                      # ragged, no prefix, an empty context
     dict(**LLAMA, l_P=200, ctx_lens=[[70, 700]]),                                  # prefix longer than a tile; 11 row blocks
+    dict(H_q=8, H_kv=8, d=64, l_P=5, ctx_lens=[[300, 17]]),                        # G = 1, d = 64
+    dict(H_q=8, H_kv=1, d=128, l_P=130, ctx_lens=[[33, 64, 65]]),                  # G = 8
 ])
 def test_encode(kw):
     b = wl.make_batch(l_q=1, seed=6, with_encode_q=True, name="encode", **kw)
     _check_encode(b)
+
+
+def test_attend_host_matches_attend():
+    """The host-buffer entry point (pinned host tensors in and out) gives the same result as the device-pointer one."""
+    b = wl.make_batch(**LLAMA, l_P=32, ctx_lens=[[256] * 6], l_q=64, seed=9, T=0.9, S=0.9, name="host")
+    ref, _, _ = gpu_attend(b, libape.APE_PREFILL, want_lse=False)
+    dev = torch.device("cuda:0")
+    q, k, v = torch.zeros_like(b.q, device=dev), torch.zeros_like(b.k_pool, device=dev), torch.zeros_like(b.v_pool, device=dev)
+    out = torch.zeros_like(q)
+    plan = handle().attend_plan(H_q=b.H_q, H_kv=b.H_kv, d=b.d, k_pool=k, v_pool=v, q=q, out=out, requests=b.requests,
+                                mode=libape.APE_PREFILL)
+    ws = plan.alloc_workspace()
+    hq, hk, hv = b.q.pin_memory(), b.k_pool.pin_memory(), b.v_pool.pin_memory()
+    hout = torch.empty_like(hq).pin_memory()
+    h2d, d2h = plan.attend_host(b.T, b.S, ws, hq, hk, hv, hout)
+    assert h2d == hq.numel() * 2 + 2 * hk.numel() * 2 and d2h == hq.numel() * 2
+    assert torch.equal(hout, ref)
+    plan.close()
