@@ -99,6 +99,18 @@ int ape_attend_plan(ape_handle_t handle, const ape_shape_t *shape, const ape_kv_
                     const ape_request_t *requests, int32_t n_req, ape_mode_t mode, ape_plan_t *plan);
 
 /*
+ * Same as ape_attend_plan, for the per-context form of the appendix "Hierarchical Formula for APE" (Eq. 11-12): every
+ * context C_i keeps its own softmax and enters the final merge with S * LogSumExp_i, i.e. the context mass is
+ * sum_i Z_i^S instead of Eq. 5's (sum_i Z_i)^S.  The two forms agree when S = 1 or when there is one context; this
+ * form depends on the context boundaries (contexts are never fused), and is the building block of the
+ * tree-structured merge the paper names as a future direction.  Launch with ape_attend as usual.  Work items are
+ * cut at every context boundary, so this form is slower when contexts are short.
+ */
+int ape_attend_plan_per_context(ape_handle_t handle, const ape_shape_t *shape, const ape_kv_pool_t *pool,
+                                const ape_rows_t *q, const ape_rows_t *out, float *lse,
+                                const ape_request_t *requests, int32_t n_req, ape_mode_t mode, ape_plan_t *plan);
+
+/*
  * Plan the block-diagonal encoding of n_ctx contexts against one shared prefix.  `q` and `out` are aligned
  * with the pool: row t belongs to pool token t (only rows inside the context spans are read / written).
  * `lse` (nullable, fp32 [pool rows, H_q]) receives each row's log-sum-exp.

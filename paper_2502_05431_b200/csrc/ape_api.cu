@@ -53,6 +53,7 @@ struct ape_plan_s {
     int64_t max_kv_extra = 0;
     CUtensorMap tm_q{}, tm_k{}, tm_v{};
     int32_t last_launches = 0;
+    bool per_context = false;        // merge form: Eq. 5 (false) or Eq. 11-12 (true)
 };
 
 namespace {
@@ -135,6 +136,25 @@ std::vector<ape_span_t> fuse_spans(const ape_span_t* ctx, int n) {
     return out;
 }
 
+// Tile ranges of the context segment: one range over the fused spans (Eq. 5 form), or one range per non-empty
+// context in the caller's order (per-context form).
+std::vector<std::pair<int, int>> add_context_tiles(std::vector<DevTile>& tiles, const ape_span_t* ctx, int n, int tile, bool per_context) {
+    std::vector<std::pair<int, int>> ranges;
+    if (!per_context) {
+        const int t0 = static_cast<int>(tiles.size());
+        for (const auto& s : fuse_spans(ctx, n)) add_span_tiles(tiles, s.start, s.len, tile, 0, 0);
+        if (static_cast<int>(tiles.size()) > t0) ranges.push_back({t0, static_cast<int>(tiles.size())});
+    } else {
+        for (int i = 0; i < n; ++i) {
+            if (ctx[i].len <= 0) continue;
+            const int t0 = static_cast<int>(tiles.size());
+            add_span_tiles(tiles, ctx[i].start, ctx[i].len, tile, 0, 0);
+            ranges.push_back({t0, static_cast<int>(tiles.size())});
+        }
+    }
+    return ranges;
+}
+
 struct HostMeta {
     std::vector<DevTile> tiles;
     std::vector<DevItem> items;
@@ -145,6 +165,7 @@ struct HostMeta {
 
 struct Run {   // a run of tiles of one segment for one (request, kv head, row-block group)
     int req, kv_head, row_block, n_sib, seg, t0, t1, merge0;
+    int ctx_id = 0;   // per-context plans: ordinal of the context of a SEG_CTX run
 };
 
 // Split the concatenation of all runs evenly over n_bins bins (each bin = one CTA or one sibling group);
@@ -163,7 +184,7 @@ void assign_stream(const std::vector<Run>& runs, int n_bins, int slot_mult, Host
             it.req = r.req; it.kv_head = r.kv_head; it.row_block = r.row_block;
             it.tile_begin = t; it.tile_end = t + take;
             it.slot = static_cast<int32_t>(m.items.size()) * slot_mult;
-            it.seg = r.seg; it.n_sib = r.n_sib;
+            it.seg = r.seg; it.n_sib = r.n_sib; it.ctx_id = r.ctx_id;
             // bookkeeping for the merge: every live sibling's group record learns about this partial
             for (int s = 0; s < r.n_sib; ++s) {
                 DevMerge& g = m.merge[r.merge0 + s];
@@ -183,7 +204,7 @@ void assign_stream(const std::vector<Run>& runs, int n_bins, int slot_mult, Host
 void finish_items(HostMeta& m) {
     for (auto& it : m.items) {
         const DevReq& rq = m.reqs[it.req];
-        it.q_row0 = rq.q_row0; it.q_len = rq.q_len; it.l_k = rq.l_k; it.pad = 0;
+        it.q_row0 = rq.q_row0; it.q_len = rq.q_len; it.l_k = rq.l_k;
         if (it.tile_begin < static_cast<int32_t>(m.tiles.size())) it.first_tile = m.tiles[it.tile_begin];
         else it.first_tile = DevTile{0, 0, 0, 0};
     }
@@ -265,9 +286,9 @@ int ape_plan_destroy(ape_plan_t p) {
     return APE_OK;
 }
 
-int ape_attend_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
-                    const ape_rows_t* out, float* lse, const ape_request_t* reqs, int32_t n_req, ape_mode_t mode,
-                    ape_plan_t* plan_out)
+static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
+                            const ape_rows_t* out, float* lse, const ape_request_t* reqs, int32_t n_req, ape_mode_t mode,
+                            bool per_context, ape_plan_t* plan_out)
 {
     if (!h || !plan_out) return APE_ERR_INVALID_ARG;
     *plan_out = nullptr;
@@ -296,7 +317,7 @@ int ape_attend_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
     ape_plan_t p = new (std::nothrow) ape_plan_s();
     if (!p) return APE_ERR_NOMEM;
     p->h = h; p->kind = (mode == APE_DECODE) ? PLAN_DECODE : PLAN_PREFILL;
-    p->shape = *shape; p->c = c; p->G = G; p->pool = *pool; p->q = *q; p->out = *out; p->lse = lse;
+    p->shape = *shape; p->c = c; p->G = G; p->pool = *pool; p->q = *q; p->out = *out; p->lse = lse; p->per_context = per_context;
     p->max_kv_extra = (mode == APE_DECODE) ? max_extra : 0;
     const int D = shape->head_dim, H_kv = shape->n_kv_heads;
 
@@ -315,14 +336,14 @@ int ape_attend_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
                 add_span_tiles(m.tiles, rq.prefix.start, rq.prefix.len, tile, 0, 0);
                 add_span_tiles(m.tiles, rq.query_kv.start, rq.query_kv.len, tile, TILE_GROWS, rq.query_kv_capacity);
                 const int o1 = static_cast<int>(m.tiles.size());
-                for (const auto& s : fuse_spans(rq.ctx, rq.n_ctx)) add_span_tiles(m.tiles, s.start, s.len, tile, 0, 0);
-                const int c1 = static_cast<int>(m.tiles.size());
+                const auto ctx_ranges = add_context_tiles(m.tiles, rq.ctx, rq.n_ctx, tile, per_context);
                 for (int hh = 0; hh < H_kv; ++hh) {
                     DevMerge g{r, hh, 0, 0, 0, 0, 0, 1};
                     const int mi = static_cast<int>(m.merge.size());
                     m.merge.push_back(g);
                     runs.push_back(Run{r, hh, 0, 1, SEG_OTHER, o0, o1, mi});
-                    if (c1 > o1) runs.push_back(Run{r, hh, 0, 1, SEG_CTX, o1, c1, mi});
+                    for (size_t ci = 0; ci < ctx_ranges.size(); ++ci)
+                        runs.push_back(Run{r, hh, 0, 1, SEG_CTX, ctx_ranges[ci].first, ctx_ranges[ci].second, mi, static_cast<int>(ci)});
                 }
             }
             p->n_cta = h->n_sm;
@@ -351,8 +372,7 @@ int ape_attend_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
                 add_span_tiles(m.tiles, rq.prefix.start, rq.prefix.len, tile, 0, 0);
                 add_span_tiles(m.tiles, rq.query_kv.start, rq.query_kv.len, tile, TILE_CAUSAL, 0);
                 const int o1 = static_cast<int>(m.tiles.size());
-                for (const auto& s : fuse_spans(rq.ctx, rq.n_ctx)) add_span_tiles(m.tiles, s.start, s.len, tile, 0, 0);
-                const int c1 = static_cast<int>(m.tiles.size());
+                const auto ctx_ranges = add_context_tiles(m.tiles, rq.ctx, rq.n_ctx, tile, per_context);
                 const int RB = static_cast<int>((rq.q_len + TB - 1) / TB);
                 for (int hh = 0; hh < H_kv; ++hh) {
                     for (int rb0 = 0; rb0 < RB; rb0 += p->n_sib) {
@@ -360,7 +380,8 @@ int ape_attend_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
                         const int mi = static_cast<int>(m.merge.size());
                         for (int s = 0; s < live; ++s) m.merge.push_back(DevMerge{r, hh, rb0 + s, 0, 0, 0, 0, 1});
                         runs.push_back(Run{r, hh, rb0, live, SEG_OTHER, o0, o1, mi});
-                        if (c1 > o1) runs.push_back(Run{r, hh, rb0, live, SEG_CTX, o1, c1, mi});
+                        for (size_t ci = 0; ci < ctx_ranges.size(); ++ci)
+                            runs.push_back(Run{r, hh, rb0, live, SEG_CTX, ctx_ranges[ci].first, ctx_ranges[ci].second, mi, static_cast<int>(ci)});
                     }
                 }
             }
@@ -382,6 +403,20 @@ int ape_attend_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
     if (rc) { ape_plan_destroy(p); return rc; }
     *plan_out = p;
     return APE_OK;
+}
+
+int ape_attend_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
+                    const ape_rows_t* out, float* lse, const ape_request_t* reqs, int32_t n_req, ape_mode_t mode,
+                    ape_plan_t* plan_out)
+{
+    return attend_plan_impl(h, shape, pool, q, out, lse, reqs, n_req, mode, false, plan_out);
+}
+
+int ape_attend_plan_per_context(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
+                                const ape_rows_t* out, float* lse, const ape_request_t* reqs, int32_t n_req, ape_mode_t mode,
+                                ape_plan_t* plan_out)
+{
+    return attend_plan_impl(h, shape, pool, q, out, lse, reqs, n_req, mode, true, plan_out);
 }
 
 int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
@@ -506,7 +541,7 @@ int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace
     p->last_launches++;
 
     MergeParams mp;
-    mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.n_groups = p->n_merge; mp.rows_per_slot = rows_per_slot;
+    mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.items = p->d_items; mp.per_context = p->per_context ? 1 : 0; mp.n_groups = p->n_merge; mp.rows_per_slot = rows_per_slot;
     mp.tokens_per_block = rows_per_slot / G; mp.ws_o = ws_o; mp.ws_ml = ws_ml; mp.out = rows_desc(p->out); mp.lse_out = p->lse;
     mp.S = S; mp.G = G; mp.H_q = p->shape.n_q_heads; mp.D = D;
     if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;
@@ -681,13 +716,12 @@ int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, cons
             add_span_tiles(m.tiles, rq.prefix.start, rq.prefix.len, tile, 0, 0);
             add_span_tiles(m.tiles, rq.query_kv.start, rq.query_kv.len, tile, TILE_GROWS, rq.query_kv_capacity);
             const int o1 = static_cast<int>(m.tiles.size());
-            for (const auto& sp : fuse_spans(rq.ctx, rq.n_ctx)) add_span_tiles(m.tiles, sp.start, sp.len, tile, 0, 0);
-            const int c1 = static_cast<int>(m.tiles.size());
+            const auto ctx_ranges = add_context_tiles(m.tiles, rq.ctx, rq.n_ctx, tile, false);
             for (int hh = 0; hh < H_kv; ++hh) {
                 const int mi = static_cast<int>(m.merge.size());
                 m.merge.push_back(DevMerge{r, hh, 0, 0, 0, 0, 0, 1});
                 runs.push_back(Run{r, hh, 0, 1, SEG_OTHER, o0, o1, mi});
-                if (c1 > o1) runs.push_back(Run{r, hh, 0, 1, SEG_CTX, o1, c1, mi});
+                for (const auto& cr : ctx_ranges) runs.push_back(Run{r, hh, 0, 1, SEG_CTX, cr.first, cr.second, mi});
             }
         }
         assign_stream(runs, n_cta, 1, m);
@@ -741,7 +775,7 @@ int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, cons
     dp.kv_extra = static_cast<int32_t>(kv_extra); dp.G = G; dp.n_stages = n_stages; dp.status = reinterpret_cast<int*>(base);
     if (launch_decode(D, tm_k, tm_v, dp, n_cta, smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
     MergeParams mp;
-    mp.groups = reinterpret_cast<const DevMerge*>(base + o_merge); mp.reqs = dp.reqs; mp.n_groups = static_cast<int32_t>(m.merge.size());
+    mp.groups = reinterpret_cast<const DevMerge*>(base + o_merge); mp.reqs = dp.reqs; mp.items = dp.items; mp.per_context = 0; mp.n_groups = static_cast<int32_t>(m.merge.size());
     mp.rows_per_slot = G; mp.tokens_per_block = 1; mp.ws_o = ws_o; mp.ws_ml = ws_ml; mp.out = rows_desc(*out); mp.lse_out = lse;
     mp.S = S; mp.G = G; mp.H_q = shape->n_q_heads; mp.D = D;
     if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;

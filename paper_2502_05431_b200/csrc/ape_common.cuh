@@ -35,7 +35,7 @@ struct DevItem {
     int32_t q_row0;      // first row of Q / O of the request (encode: context start)
     int32_t q_len;       // query rows of the request
     int32_t l_k;         // keys in the query segment at planning time (encode: context length)
-    int32_t pad;
+    int32_t ctx_id;      // SEG_CTX items of a per-context plan: ordinal of the context the tiles belong to, else 0
     DevTile first_tile;  // tiles[tile_begin]
 };
 static_assert(sizeof(DevItem) == 64, "DevItem is one 64-byte record");

@@ -39,6 +39,58 @@ __device__ __forceinline__ void combine_segment(const float* __restrict__ ws_o, 
     }
 }
 
+// Per-context form (appendix "Hierarchical Formula for APE", Eq. 11-12): every context C_i keeps its own normalised
+// output and enters the final softmax with S * LSE_i.  Partials arrive grouped by context (consecutive slots with the same
+// context ordinal); the result is the context segment's normalised output `acc` (to be divided by `norm`) and its
+// scaled base-2 log weight `lse` = log2 sum_i 2^(S * LSE_i).
+template <int VEC>
+__device__ __forceinline__ void combine_per_context(const MergeParams& p, const DevMerge& g, int row, int lane,
+                                                    float& lse, float& norm, float (&acc)[VEC])
+{
+    float top = -INFINITY, Z = 0.f;                   // running maximum of S * LSE_i and sum of 2^(S * LSE_i - top)
+    #pragma unroll
+    for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
+    float M = -INFINITY, L = 0.f, a[VEC];
+    #pragma unroll
+    for (int v = 0; v < VEC; ++v) a[v] = 0.f;
+    const int item0 = g.ctx_slot0 / g.slot_stride;
+    int cur = (g.ctx_n > 0) ? p.items[item0].ctx_id : 0;
+    auto fold = [&]() {                               // close the current context
+        if (L > 0.f) {
+            const float li = p.S * (M + fast_log2(L));
+            const float tn = fmaxf(top, li);
+            const float f_old = fast_exp2(top - tn), f_new = fast_exp2(li - tn) / L;
+            #pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[v] = acc[v] * f_old + a[v] * f_new;
+            Z = Z * f_old + fast_exp2(li - tn);
+            top = tn;
+        }
+        M = -INFINITY; L = 0.f;
+        #pragma unroll
+        for (int v = 0; v < VEC; ++v) a[v] = 0.f;
+    };
+    for (int i = 0; i < g.ctx_n; ++i) {
+        const int cid = p.items[item0 + i].ctx_id;
+        if (cid != cur) { fold(); cur = cid; }
+        const size_t slot = static_cast<size_t>(g.ctx_slot0) + static_cast<size_t>(i) * g.slot_stride;
+        const float2 ml = *reinterpret_cast<const float2*>(p.ws_ml + (slot * p.rows_per_slot + row) * 2);
+        if (!(ml.y > 0.f)) continue;
+        const float Mn = fmaxf(M, ml.x);
+        const float f_old = fast_exp2(M - Mn), f_new = fast_exp2(ml.x - Mn);
+        const float* src = p.ws_o + (slot * p.rows_per_slot + row) * p.D + lane * VEC;
+        float x[VEC];
+        if constexpr (VEC == 4) { const float4 t = *reinterpret_cast<const float4*>(src); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
+        else { const float2 t = *reinterpret_cast<const float2*>(src); x[0] = t.x; x[1] = t.y; }
+        #pragma unroll
+        for (int v = 0; v < VEC; ++v) a[v] = a[v] * f_old + x[v] * f_new;
+        L = L * f_old + ml.y * f_new;
+        M = Mn;
+    }
+    fold();
+    norm = Z;
+    lse = (Z > 0.f) ? top + fast_log2(Z) : -INFINITY;
+}
+
 template <int VEC>
 __global__ void __launch_bounds__(256) ape_merge_kernel(const MergeParams p)
 {
@@ -54,11 +106,16 @@ __global__ void __launch_bounds__(256) ape_merge_kernel(const MergeParams p)
     if (tok >= rq.q_len) return;
 
     float Mc, Lc, Mo, Lo, ac[VEC], ao[VEC];
-    combine_segment<VEC>(p.ws_o, p.ws_ml, g.ctx_slot0, g.ctx_n, g.slot_stride, p.rows_per_slot, row, p.D, lane, Mc, Lc, ac);
+    float lse_c;
+    if (p.per_context) {
+        combine_per_context<VEC>(p, g, row, lane, lse_c, Lc, ac);      // Lc: the normaliser of ac
+    } else {
+        combine_segment<VEC>(p.ws_o, p.ws_ml, g.ctx_slot0, g.ctx_n, g.slot_stride, p.rows_per_slot, row, p.D, lane, Mc, Lc, ac);
+        // base-2 log-sum-exp of the context segment, multiplied by S (Eq. 5: Z_C^S)
+        lse_c = (Lc > 0.f) ? p.S * (Mc + fast_log2(Lc)) : -INFINITY;
+    }
     combine_segment<VEC>(p.ws_o, p.ws_ml, g.oth_slot0, g.oth_n, g.slot_stride, p.rows_per_slot, row, p.D, lane, Mo, Lo, ao);
 
-    // base-2 log-sum-exps of the two segments; the context one is multiplied by S (Eq. 5: Z_C^S)
-    const float lse_c = (Lc > 0.f) ? p.S * (Mc + fast_log2(Lc)) : -INFINITY;
     const float lse_o = (Lo > 0.f) ? (Mo + fast_log2(Lo)) : -INFINITY;
     const float top = fmaxf(lse_c, lse_o);
     float wc = 0.f, wo = 0.f, lam = -INFINITY;

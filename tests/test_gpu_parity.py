@@ -204,3 +204,35 @@ def test_attend_host_matches_attend():
     assert h2d == hq.numel() * 2 + 2 * hk.numel() * 2 and d2h == hq.numel() * 2
     assert torch.equal(hout, ref)
     plan.close()
+
+
+# ---- per-context form (Eq. 11-12) -------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("mode,kw", [
+    (libape.APE_PREFILL, dict(**LLAMA, l_P=32, ctx_lens=[[256] * 10], l_q=64, T=0.9, S=0.7)),
+    (libape.APE_PREFILL, dict(**LLAMA, l_P=7, ctx_lens=[[130, 1, 255, 0, 40], [77]], l_q=33, l_k=50, gap=5, T=0.6, S=0.5, shuffle_ctx=True)),
+    (libape.APE_PREFILL, dict(H_q=4, H_kv=1, d=64, l_P=16, ctx_lens=[[64] * 4], l_q=16, T=0.8, S=0.9)),
+    (libape.APE_DECODE, dict(**LLAMA, l_P=5, ctx_lens=[[70, 1, 129], [200, 300, 64, 64]], l_q=1, l_k=3, gap=3, T=0.7, S=0.6)),
+    (libape.APE_DECODE, dict(**LLAMA, l_P=64, ctx_lens=[[256] * 40], l_q=1, l_k=100, T=0.9, S=0.8)),
+])
+def test_per_context_form(mode, kw):
+    """S on every context's own log-sum-exp: checked against the oracle's per-context switch; differs from Eq. 5."""
+    b = wl.make_batch(seed=11, name="per_context", **kw)
+    out, lse, _ = gpu_attend(b, mode, per_context=True)
+    flat, _, _ = gpu_attend(b, mode)
+    differs = False
+    for r, rq in enumerate(b.requests):
+        q, p, c, k = b.views(r)
+        ref = orc.attend(q, p, c, k, b.T, b.S, per_context=True)
+        sl = slice(rq.q_start, rq.q_start + rq.q_len)
+        compare(out[sl], ref.out.float(), f"per-context req {r}")
+        assert (lse[sl].double() - ref.lse).abs().max().item() < 2e-3
+        differs |= (out[sl].float() - flat[sl].float()).abs().max().item() > 1e-3
+    assert differs, "the per-context form should not coincide with Eq. 5 here (several contexts, S != 1)"
+
+
+def test_per_context_form_with_one_context_equals_flat():
+    b = wl.make_batch(**LLAMA, l_P=20, ctx_lens=[[700]], l_q=40, seed=12, T=0.8, S=0.6, name="one_ctx")
+    a, _, _ = gpu_attend(b, libape.APE_PREFILL, per_context=True)
+    f, _, _ = gpu_attend(b, libape.APE_PREFILL)
+    assert (a.float() - f.float()).abs().max().item() <= 2e-2
