@@ -4,6 +4,7 @@ enough that a multi-pass capture ends by itself.
     python -m paper_2502_05431_b200.profile_case prefill|decode|encode [--iters 3]
 
 prefill: 256 query rows over prefix 64 + 250 x 256 context tokens (KV 262 MB), Llama-3-8B head shape.
+rag    : 4 requests x 20 contexts of 512..1536 tokens, 128 query rows each (KV 339 MB).
 decode : 4 requests x (64 + 250 x 256 + 257) cached tokens (KV 1.05 GB), one new token each.
 encode : 250 contexts x 256 tokens against a 64-token prefix.
 Prints the CUDA-event time per launch pair and the algorithmic work, so that a capture can be scaled.
@@ -20,14 +21,24 @@ from . import libape, workloads as wl
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["prefill", "decode", "encode"])
+    ap.add_argument("case", choices=["prefill", "decode", "encode", "rag"])
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--n-ctx", type=int, default=250)
     args = ap.parse_args()
     dev = "cuda:0"
     h = libape.Handle(0)
     H_q, H_kv, d = 32, 8, 128
-    if args.case == "decode":
+    if args.case == "rag":
+        # RAG shape: 4 independent requests, 20 contexts of 512..1536 tokens each, 128 query rows (config 3)
+        lens = wl.config3_lens(0)
+        b = wl.make_batch(H_q=H_q, H_kv=H_kv, d=d, l_P=64, ctx_lens=lens, l_q=128, seed=0, T=0.9, S=0.8, device=dev)
+        out = torch.zeros_like(b.q)
+        plan = h.attend_plan(H_q=H_q, H_kv=H_kv, d=d, k_pool=b.k_pool, v_pool=b.v_pool, q=b.q, out=out, requests=b.requests,
+                             mode=libape.APE_PREFILL)
+        ws = plan.alloc_workspace()
+        run = lambda: plan.attend(b.T, b.S, ws)
+        work = {"flops": sum(4.0 * d * H_q * (128 * (64 + sum(l)) + 128 * 129 / 2) for l in lens)}
+    elif args.case == "decode":
         b = wl.config5(n_req=4, n_ctx=args.n_ctx, steps=8, device=dev)
         q = b.extra["q_steps"][0].contiguous()
         out = torch.zeros_like(q)

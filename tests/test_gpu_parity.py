@@ -236,3 +236,15 @@ def test_per_context_form_with_one_context_equals_flat():
     a, _, _ = gpu_attend(b, libape.APE_PREFILL, per_context=True)
     f, _, _ = gpu_attend(b, libape.APE_PREFILL)
     assert (a.float() - f.float()).abs().max().item() <= 2e-2
+
+
+def test_prefill_long_query_many_row_blocks():
+    """1,500 causal query rows (24 row blocks, six sibling groups) over a modest context: sampled rows against the oracle."""
+    b = wl.make_batch(**LLAMA, l_P=64, ctx_lens=[[700, 300]], l_q=1500, l_k=1600, seed=13, T=0.9, S=0.9, name="long_q")
+    out, lse, _ = gpu_attend(b, libape.APE_PREFILL)
+    assert not torch.isnan(out.float()).any()
+    for rows in [(0, 3), (63, 66), (700, 703), (1497, 1500)]:
+        ref = oracle_attend(b, 0, rows=rows)
+        compare(out, ref.out.float(), f"long_q rows {rows}")
+        sel = ~torch.isnan(ref.lse)
+        assert (lse.double()[sel] - ref.lse[sel]).abs().max().item() < 2e-3
