@@ -51,7 +51,8 @@ struct ape_plan_s {
     size_t smem_bytes = 0;
     size_t ws_bytes = 0;
     int64_t max_kv_extra = 0;
-    CUtensorMap tm_q{}, tm_k{}, tm_v{};
+    CUtensorMap tm_q{}, tm_k{}, tm_v{}, tm_o{};
+    bool o_via_tma = false;         // encode plans: tm_o describes the output rows
     int32_t last_launches = 0;
     bool per_context = false;        // merge form: Eq. 5 (false) or Eq. 11-12 (true)
 };
@@ -485,6 +486,9 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
         rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
         if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
         if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
+        // Every item of this plan has a row block of its own, so a finished row block may leave through its Q buffer.
+        if (!rc) p->o_via_tma = make_map(h, &p->tm_o, out->data, D, shape->n_q_heads, out->n_rows, out->head_stride, out->token_stride,
+                                         G, 128 / G) == APE_OK;
         if (!rc && attn_set_smem_attr(D, 2, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
         if (!rc) { finish_items(m); rc = upload(p, m); }
     } catch (const std::bad_alloc&) {
@@ -536,7 +540,8 @@ int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace
         ap.out = rows_desc(p->out); ap.lse_out = nullptr; ap.ws_o = ws_o; ap.ws_ml = ws_ml;
         ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c / T * kLog2e;
         ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = p->n_sib; ap.n_q_bufs = 1; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
-        if (launch_attn(D, p->tm_q, p->tm_k, p->tm_v, ap, p->n_cta, p->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
+        ap.o_via_tma = 0;
+        if (launch_attn(D, p->tm_q, p->tm_k, p->tm_v, p->tm_q, ap, p->n_cta, p->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
     }
     p->last_launches++;
 
@@ -562,7 +567,8 @@ int ape_encode_contexts(ape_plan_t p, void* workspace, size_t ws_bytes, void* st
     ap.out = rows_desc(p->out); ap.lse_out = p->lse; ap.ws_o = nullptr; ap.ws_ml = nullptr;
     ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c * kLog2e;
     ap.G = p->G; ap.H_q = p->shape.n_q_heads; ap.n_sib = 1; ap.n_q_bufs = 2; ap.q_rows_are_pool = 1; ap.status = p->h->d_status;
-    if (launch_attn(p->shape.head_dim, p->tm_q, p->tm_k, p->tm_v, ap, p->n_cta, p->smem_bytes,
+    ap.o_via_tma = p->o_via_tma ? 1 : 0;
+    if (launch_attn(p->shape.head_dim, p->tm_q, p->tm_k, p->tm_v, p->tm_o, ap, p->n_cta, p->smem_bytes,
                     static_cast<cudaStream_t>(stream_v)) != cudaSuccess) return APE_ERR_CUDA;
     p->last_launches = 1;
     return APE_OK;

@@ -80,7 +80,7 @@ __device__ __forceinline__ bool tile_visible(const DevTile& t, const ItemGeom& g
 template <int D, int QBUF>
 __global__ void __launch_bounds__(kThreads, 1)
 ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const AttnParams p)
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const AttnParams p)
 {
     constexpr int kSlabs = D / 64;
     constexpr int kTileBytes = kSlabs * kSlabBytes;            // one K or V tile, also one Q half
@@ -107,6 +107,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t bar_o_full = bar_p_full + 64;               // [2]
     const uint32_t bar_done = bar_o_full + 16;
     const uint32_t bar_tok = bar_done + 8;                     // [2]: turn-taking of the two halves' exponential phases
+    const uint32_t bar_o_staged = bar_tok + 16;                // [2]: a half's O tile sits in shared memory, ready for its bulk store
     __shared__ uint32_t tmem_base_smem;
     __shared__ int abort_flag;
 
@@ -124,6 +125,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         mbar_init(bar_done, 2);
         mbar_init(bar_tok, 4); mbar_init(bar_tok + 8, 4);          // one arrival per softmax warp of the other half
+        mbar_init(bar_o_staged, 4); mbar_init(bar_o_staged + 8, 4);  // one arrival per softmax warp of the half
         mbar_fence_init();
     }
     if (warp == kMmaWarp) {
@@ -148,6 +150,12 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         g.off = rq.l_k - rq.q_len;
         return g;
     };
+
+    // A half whose 128 rows are all live query rows can leave as one tile (bulk store); ragged halves are written row by row.
+    auto half_is_full = [&](const DevReq& rq, const ItemGeom& g, int w) {
+        return g.rb * TB + (w + 1) * (kHalfRows / G) <= rq.q_len;
+    };
+    const bool o_via_tma = (QBUF == 2) && p.o_via_tma != 0;
 
     // Register hand-over at the head of every role: the softmax threads hold a whole 128-column row of S in registers,
     // the third warpgroup (producer, MMA issuers, one idle warp) gives its share up.
@@ -400,7 +408,8 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t tS = tmem_base + lane_base + (w ? kColS1 : kColS0);
         const uint32_t tO = tmem_base + lane_base + (w ? kColO1 : kColO0);
         const uint32_t my_s_full = bar_s_full + 8 * w, my_p_full = bar_p_full + 32 * w, my_o_full = bar_o_full + 8 * w;
-        uint32_t scnt = 0, ocnt = 0;
+        uint32_t scnt = 0, ocnt = 0, q_loads = 0;
+        int last_req = -1, last_head = -1, last_rb = -1;
         bool ok = true;
 
         for (int it = item_begin; it < item_end && ok; ++it) {
@@ -409,6 +418,9 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (sib >= item.n_sib) continue;
             const DevReq rq{item.q_row0, item.q_len, item.l_k, 0};
             const ItemGeom g = geom(item, rq);
+            if (!(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
+                ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
+            }
             const int tok = g.rb * TB + R / G;
             const int hg = R % G;
             const bool live = tok < rq.q_len;
@@ -530,6 +542,30 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 __nv_bfloat16* dst = p.out.data + static_cast<int64_t>(rq.q_row0 + tok) * p.out.token_stride
                                      + static_cast<int64_t>(h) * p.out.head_stride;
                 const bool wide_ok = (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;
+                if (o_via_tma && half_is_full(rq, g, w)) {
+                    // The item's Q buffer is free (O is final, so every S = Q K^T that read it is done) and has the layout
+                    // the bulk store wants: row r of the half, 16-byte chunk j of a 128-byte line at chunk j ^ (r mod 8).
+                    uint8_t* stage = q_smem + ((q_loads - 1) % QBUF) * kQBytes + w * kTileBytes + r_local * 128;
+                    #pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c * 32, o);
+                        tmem_ld_wait();
+                        #pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint4 v;
+                            v.x = pack_bf16x2(__uint_as_float(o[8 * j + 0]) * inv, __uint_as_float(o[8 * j + 1]) * inv);
+                            v.y = pack_bf16x2(__uint_as_float(o[8 * j + 2]) * inv, __uint_as_float(o[8 * j + 3]) * inv);
+                            v.z = pack_bf16x2(__uint_as_float(o[8 * j + 4]) * inv, __uint_as_float(o[8 * j + 5]) * inv);
+                            v.w = pack_bf16x2(__uint_as_float(o[8 * j + 6]) * inv, __uint_as_float(o[8 * j + 7]) * inv);
+                            const int chunk = (c & 1) * 4 + j;
+                            *reinterpret_cast<uint4*>(stage + (c >> 1) * kSlabBytes + ((chunk ^ (r_local & 7)) << 4)) = v;
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_o_staged + 8 * w);
+                } else
                 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t o[32];
@@ -581,9 +617,31 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
         if (QBUF == 2 && lane == 0) {
             tma_prefetch_desc(&tm_q);
-            uint32_t q_loads = 0;
+            if (o_via_tma) tma_prefetch_desc(&tm_o);
+            uint32_t q_loads = 0, staged[2] = {0, 0};
             int last_req = -1, last_head = -1, last_rb = -1;
             bool ok = true;
+            // what the bulk store of a row block needs, kept for the two row blocks whose buffers are in use
+            struct Pending { int head0, tok0; bool full[2]; } pend[2] = {{0, 0, {false, false}}, {0, 0, {false, false}}};
+            // O of the row block that used buffer qb: wait for each staged half, send it, and return once the copies have
+            // read the buffer (it is about to be refilled with the next Q).
+            auto drain = [&](uint32_t qb) {
+                bool any = false;
+                #pragma unroll
+                for (int w = 0; w < 2; ++w) {
+                    if (!pend[qb].full[w]) continue;
+                    if (!mbar_wait(bar_o_staged + 8 * w, staged[w] & 1, &abort_flag, p.status)) return false;
+                    ++staged[w];
+                    #pragma unroll
+                    for (int sl = 0; sl < kSlabs; ++sl)
+                        tma_store_3d(&tm_o, smem_u32(q_smem + qb * kQBytes + w * kTileBytes + sl * kSlabBytes),
+                                     sl * 64, pend[qb].head0, pend[qb].tok0 + w * (kHalfRows / G));
+                    any = true;
+                }
+                if (any) { bulk_commit_group(); bulk_wait_read_all(); }
+                pend[qb].full[0] = pend[qb].full[1] = false;
+                return true;
+            };
             for (int it = item_begin; it < item_end && ok; ++it) {
                 const DevItem item = p.items[it];
                 if (it + 1 < item_end) prefetch_l1(&p.items[it + 1]);   // the next item's record is in cache when its turn comes
@@ -591,8 +649,17 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const DevReq rq{item.q_row0, item.q_len, item.l_k, 0};
                 const ItemGeom g = geom(item, rq);
                 if (item.req == last_req && item.kv_head == last_head && g.rb == last_rb) continue;
+                const uint32_t qb = q_loads % QBUF;
+                if (o_via_tma && !drain(qb)) { ok = false; break; }
                 if (!load_q(item, rq, g, q_loads)) { ok = false; break; }
+                if (o_via_tma && item.seg == SEG_FINAL) {
+                    pend[qb].head0 = item.kv_head * G; pend[qb].tok0 = rq.q_row0 + g.rb * TB;
+                    pend[qb].full[0] = half_is_full(rq, g, 0); pend[qb].full[1] = half_is_full(rq, g, 1);
+                }
                 ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
+            }
+            if (ok && o_via_tma) {                                  // the last two row blocks, oldest first
+                ok = drain(q_loads % QBUF) && drain((q_loads + 1) % QBUF);
             }
             if (!ok) {
                 const long long t0 = clock64();
@@ -646,13 +713,13 @@ cudaError_t attn_set_smem_attr(int D, int q_bufs, size_t smem_bytes) {
     return cudaFuncSetAttribute(ape_attn_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
 }
 
-cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const CUtensorMap& tm_o,
                         const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream)
 {
-    if (D == 128 && p.n_q_bufs == 2) ape_attn_kernel<128, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
-    else if (D == 128) ape_attn_kernel<128, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
-    else if (p.n_q_bufs == 2) ape_attn_kernel<64, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
-    else ape_attn_kernel<64, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, p);
+    if (D == 128 && p.n_q_bufs == 2) ape_attn_kernel<128, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, p);
+    else if (D == 128) ape_attn_kernel<128, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, p);
+    else if (p.n_q_bufs == 2) ape_attn_kernel<64, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, p);
+    else ape_attn_kernel<64, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, p);
     return cudaGetLastError();
 }
 
