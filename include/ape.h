@@ -182,6 +182,46 @@ int ape_decode_noalloc(const ape_shape_t *shape, const ape_kv_pool_t *pool, cons
                        const ape_rows_t *out, float *lse, const ape_request_t *requests, int32_t n_req,
                        float T, float S, int64_t kv_extra, int device, void *stream, int32_t *device_status);
 
+/*
+ * Rotary position embedding with position re-use, fused with the write into the cache (the step right before
+ * ape_encode_contexts: it makes the K, V and Q that the pre-caching attention and, later, ape_attend read).
+ *
+ * Section "Position Embedding" of the paper names the rotary embedding (Su et al.); the section "Parallel Encoding"
+ * item "Re-using Positions for Long Context" places every context in the same range of positions.  Together with the
+ * shared prefix of section "Prepending Shared Prefix" the positions of a request are: prefix 0 .. l_P-1, EVERY context
+ * l_P .. l_P+l_i-1, query l_P + max_i l_i onward.  The pairing is the half-split one of the paper's base models
+ * (component i with i + d/2, angle pos * theta^(-2i/d)).
+ *
+ * A run copies `len` rows, source row src_start+j to destination row dst_start+j, rotated for position pos0+j.
+ */
+typedef struct { int64_t src_start, dst_start, len, pos0; } ape_rope_run_t;
+
+/*
+ * The runs of one request under position re-use (HOST helper, no GPU work): source rows are packed in the order
+ * prefix, context 1..N, query K/V, starting at row `src_start`; destinations are the request's pool spans.
+ * `runs` is a HOST array of `capacity` entries; *n_runs receives the count (N + 2, empty spans included with len 0).
+ * APE_ERR_INVALID_ARG if capacity is too small or a span is malformed.
+ */
+int ape_rope_runs_for_request(const ape_request_t *request, int64_t src_start, ape_rope_run_t *runs,
+                              int32_t capacity, int32_t *n_runs);
+
+/*
+ * Plan for a set of runs (HOST array, read during the call): cuts them into work items and uploads those
+ * (cudaMalloc + blocking copy).  head_dim 64 or 128; theta > 1 is the base of the embedding (500000 for Llama-3).
+ * Every row index must fit 31 bits.  Destroy with ape_plan_destroy.
+ */
+int ape_rope_plan(ape_handle_t handle, int32_t head_dim, double theta, const ape_rope_run_t *runs, int32_t n_runs,
+                  ape_plan_t *plan);
+
+/*
+ * Apply the plan to one tensor: src and dst are bf16 [rows, n_heads, head_dim] with strides in elements (16-byte
+ * aligned, strides multiples of 8); rotate = 1 for K and Q, 0 for V (plain copy through the same runs).  src and dst
+ * must not overlap.  Asynchronous on `stream`; allocates nothing.  Rows outside the runs are not touched.
+ * APE_ERR_INVALID_ARG if a run reaches past src->n_rows or dst->n_rows.
+ */
+int ape_rope_write(ape_plan_t plan, const ape_rows_t *src, const ape_rows_t *dst, int32_t n_heads, int32_t rotate,
+                   void *stream);
+
 /* Kernels launched by the last ape_attend / ape_encode_contexts call on this plan. */
 int ape_plan_last_launches(ape_plan_t plan, int32_t *n_launches);
 

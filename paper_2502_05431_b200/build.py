@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "lib", "libape.so")
-SOURCES = ["ape_api.cu", "ape_attn.cu", "ape_decode.cu", "ape_merge.cu"]
+SOURCES = ["ape_api.cu", "ape_attn.cu", "ape_decode.cu", "ape_merge.cu", "ape_rope.cu"]
 HEADERS = ["ape_common.cuh", "ape_kernels.h", "ape_tcgen05.cuh", os.path.join("..", "..", "include", "ape.h")]
 
 

@@ -14,7 +14,7 @@ using namespace ape;
 
 namespace {
 
-enum PlanKind { PLAN_PREFILL = 0, PLAN_DECODE = 1, PLAN_ENCODE = 2 };
+enum PlanKind { PLAN_PREFILL = 0, PLAN_DECODE = 1, PLAN_ENCODE = 2, PLAN_ROPE = 3 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -55,6 +55,11 @@ struct ape_plan_s {
     bool o_via_tma = false;         // encode plans: tm_o describes the output rows
     int32_t last_launches = 0;
     bool per_context = false;        // merge form: Eq. 5 (false) or Eq. 11-12 (true)
+    // rotary-embedding plans
+    RopeChunk* d_rope_chunks = nullptr;
+    int n_rope_chunks = 0;
+    double rope_log2_theta = 0.0;
+    int64_t rope_src_rows = 0, rope_dst_rows = 0;    // one past the largest row the runs touch
 };
 
 namespace {
@@ -496,6 +501,88 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
     }
     if (rc) { ape_plan_destroy(p); return rc; }
     *plan_out = p;
+    return APE_OK;
+}
+
+int ape_rope_runs_for_request(const ape_request_t* rq, int64_t src_start, ape_rope_run_t* runs, int32_t capacity, int32_t* n_runs) {
+    if (!rq || !runs || !n_runs || src_start < 0 || rq->n_ctx < 0 || (rq->n_ctx > 0 && !rq->ctx)) return APE_ERR_INVALID_ARG;
+    if (capacity < rq->n_ctx + 2) return APE_ERR_INVALID_ARG;
+    if (rq->prefix.len < 0 || rq->prefix.start < 0 || rq->query_kv.len < 0 || rq->query_kv.start < 0) return APE_ERR_INVALID_ARG;
+    int64_t src = src_start, longest = 0;
+    int n = 0;
+    runs[n++] = ape_rope_run_t{src, rq->prefix.start, rq->prefix.len, 0};
+    src += rq->prefix.len;
+    for (int i = 0; i < rq->n_ctx; ++i) {
+        if (rq->ctx[i].len < 0 || rq->ctx[i].start < 0) return APE_ERR_INVALID_ARG;
+        runs[n++] = ape_rope_run_t{src, rq->ctx[i].start, rq->ctx[i].len, rq->prefix.len};   // every context starts after the prefix
+        src += rq->ctx[i].len;
+        longest = std::max(longest, rq->ctx[i].len);
+    }
+    runs[n++] = ape_rope_run_t{src, rq->query_kv.start, rq->query_kv.len, rq->prefix.len + longest};
+    *n_runs = n;
+    return APE_OK;
+}
+
+int ape_rope_plan(ape_handle_t h, int32_t head_dim, double theta, const ape_rope_run_t* runs, int32_t n_runs, ape_plan_t* plan_out) {
+    if (!h || !plan_out || n_runs < 0 || (n_runs > 0 && !runs)) return APE_ERR_INVALID_ARG;
+    *plan_out = nullptr;
+    if (head_dim != 64 && head_dim != 128) return APE_ERR_SHAPE;
+    if (!(theta > 1.0) || !std::isfinite(theta)) return APE_ERR_RANGE;
+    int rc = set_device(h); if (rc) return rc;
+    ape_plan_t p = new (std::nothrow) ape_plan_s();
+    if (!p) return APE_ERR_NOMEM;
+    p->h = h; p->kind = PLAN_ROPE; p->shape.head_dim = head_dim; p->rope_log2_theta = std::log2(theta);
+    try {
+        std::vector<RopeChunk> chunks;
+        constexpr int64_t kMaxRow = (1ll << 31) - 1;
+        for (int r = 0; r < n_runs && !rc; ++r) {
+            const ape_rope_run_t& run = runs[r];
+            if (run.len < 0 || run.src_start < 0 || run.dst_start < 0 || run.pos0 < 0) { rc = APE_ERR_INVALID_ARG; break; }
+            if (run.src_start + run.len > kMaxRow || run.dst_start + run.len > kMaxRow || run.pos0 + run.len > kMaxRow) { rc = APE_ERR_LAYOUT; break; }
+            p->rope_src_rows = std::max(p->rope_src_rows, run.len ? run.src_start + run.len : 0);
+            p->rope_dst_rows = std::max(p->rope_dst_rows, run.len ? run.dst_start + run.len : 0);
+            for (int64_t off = 0; off < run.len; off += kRopeChunkTokens) {
+                RopeChunk c;
+                c.src_tok = static_cast<int32_t>(run.src_start + off); c.dst_tok = static_cast<int32_t>(run.dst_start + off);
+                c.n_tok = static_cast<int32_t>(std::min<int64_t>(kRopeChunkTokens, run.len - off));
+                c.pos0 = static_cast<int32_t>(run.pos0 + off);
+                chunks.push_back(c);
+            }
+        }
+        p->n_rope_chunks = static_cast<int>(chunks.size());
+        if (!rc && !chunks.empty()) {
+            if (cudaMalloc(&p->d_blob, chunks.size() * sizeof(RopeChunk)) != cudaSuccess) rc = APE_ERR_NOMEM;
+            else if (cudaMemcpy(p->d_blob, chunks.data(), chunks.size() * sizeof(RopeChunk), cudaMemcpyHostToDevice) != cudaSuccess) rc = APE_ERR_CUDA;
+            p->d_rope_chunks = static_cast<RopeChunk*>(p->d_blob);
+        }
+    } catch (const std::bad_alloc&) {
+        rc = APE_ERR_NOMEM;
+    }
+    if (rc) { ape_plan_destroy(p); return rc; }
+    *plan_out = p;
+    return APE_OK;
+}
+
+int ape_rope_write(ape_plan_t p, const ape_rows_t* src, const ape_rows_t* dst, int32_t n_heads, int32_t rotate, void* stream_v) {
+    if (!p || !src || !dst || !src->data || !dst->data || n_heads <= 0) return APE_ERR_INVALID_ARG;
+    if (p->kind != PLAN_ROPE) return APE_ERR_MODE;
+    const int D = p->shape.head_dim;
+    for (const ape_rows_t* r : {src, dst}) {
+        if (!aligned16(r->data) || r->head_stride % 8 || r->token_stride % 8) return APE_ERR_ALIGN;
+        if (r->head_stride < D || r->token_stride < static_cast<int64_t>(n_heads - 1) * r->head_stride + D) return APE_ERR_INVALID_ARG;
+    }
+    if (p->rope_src_rows > src->n_rows || p->rope_dst_rows > dst->n_rows) return APE_ERR_INVALID_ARG;
+    int rc = set_device(p->h); if (rc) return rc;
+    p->last_launches = 0;
+    if (p->n_rope_chunks == 0) return APE_OK;
+    RopeParams rp;
+    rp.chunks = p->d_rope_chunks; rp.n_chunks = p->n_rope_chunks;
+    rp.src.data = static_cast<const __nv_bfloat16*>(src->data); rp.src.token_stride = src->token_stride; rp.src.head_stride = src->head_stride;
+    rp.dst = rows_desc(*dst);
+    rp.n_heads = n_heads; rp.rotate = rotate ? 1 : 0; rp.log2_theta = p->rope_log2_theta;
+    const int n_cta = std::max(1, std::min(p->n_rope_chunks, p->h->n_sm * 8));
+    if (launch_rope(D, rp, n_cta, static_cast<cudaStream_t>(stream_v)) != cudaSuccess) return APE_ERR_CUDA;
+    p->last_launches = 1;
     return APE_OK;
 }
 

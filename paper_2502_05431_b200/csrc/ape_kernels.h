@@ -78,4 +78,22 @@ struct MergeParams {
 };
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
 
+// Rotary embedding with position re-use, fused with the copy to its destination.
+constexpr int kRopeChunkTokens = 16;   // tokens per work item
+struct RopeChunk {
+    int32_t src_tok, dst_tok;        // first source / destination row
+    int32_t n_tok;                   // 1 .. kRopeChunkTokens
+    int32_t pos0;                    // position of the first row; the following rows count up from it
+};
+struct RopeParams {
+    const RopeChunk* chunks;
+    int32_t n_chunks;
+    struct { const __nv_bfloat16* data; int64_t token_stride, head_stride; } src;
+    RowsDesc dst;
+    int32_t n_heads;
+    int32_t rotate;                  // 0: plain copy (V), 1: rotate (K, Q)
+    double log2_theta;
+};
+cudaError_t launch_rope(int D, const RopeParams& p, int n_cta, cudaStream_t stream);
+
 }  // namespace ape

@@ -19,7 +19,8 @@ APE_PREFILL, APE_DECODE = 0, 1
 
 EXPORTS = ["ape_create", "ape_destroy", "ape_attend_plan", "ape_encode_plan", "ape_plan_workspace_bytes",
            "ape_plan_destroy", "ape_attend", "ape_encode_contexts", "ape_attend_host", "ape_plan_last_launches",
-           "ape_get_status", "ape_status_string", "ape_decode_noalloc", "ape_attend_plan_per_context"]
+           "ape_get_status", "ape_status_string", "ape_decode_noalloc", "ape_attend_plan_per_context",
+           "ape_rope_runs_for_request", "ape_rope_plan", "ape_rope_write"]
 
 
 class ApeError(RuntimeError):
@@ -47,6 +48,10 @@ class ape_rows_t(C.Structure):
 class ape_request_t(C.Structure):
     _fields_ = [("q_start", C.c_int64), ("q_len", C.c_int64), ("prefix", ape_span_t), ("ctx", C.POINTER(ape_span_t)),
                 ("n_ctx", C.c_int32), ("query_kv", ape_span_t), ("query_kv_capacity", C.c_int64)]
+
+
+class ape_rope_run_t(C.Structure):
+    _fields_ = [("src_start", C.c_int64), ("dst_start", C.c_int64), ("len", C.c_int64), ("pos0", C.c_int64)]
 
 
 _lib = None
@@ -80,6 +85,10 @@ def load() -> C.CDLL:
         lib.ape_decode_noalloc.argtypes = [C.POINTER(ape_shape_t), C.POINTER(ape_kv_pool_t), C.POINTER(ape_rows_t),
                                            C.POINTER(ape_rows_t), vp, C.POINTER(ape_request_t), C.c_int32, C.c_float, C.c_float,
                                            C.c_int64, C.c_int, vp, C.POINTER(C.c_int32)]
+        lib.ape_rope_runs_for_request.argtypes = [C.POINTER(ape_request_t), C.c_int64, C.POINTER(ape_rope_run_t), C.c_int32,
+                                                  C.POINTER(C.c_int32)]
+        lib.ape_rope_plan.argtypes = [vp, C.c_int32, C.c_double, C.POINTER(ape_rope_run_t), C.c_int32, C.POINTER(vp)]
+        lib.ape_rope_write.argtypes = [vp, C.POINTER(ape_rows_t), C.POINTER(ape_rows_t), C.c_int32, C.c_int32, vp]
         lib.ape_status_string.argtypes = [C.c_int]
         lib.ape_status_string.restype = C.c_char_p
         for name in EXPORTS:
@@ -202,6 +211,45 @@ class Handle:
                                       lse.data_ptr() if lse is not None else None, C.byref(pre), spans, len(ctx), C.byref(p)),
                "ape_encode_plan")
         return Plan(self, p, (q, out, k_pool, v_pool, lse))
+
+
+def rope_runs_for_request(request, src_start: int = 0):
+    """ape_rope_runs_for_request: [(src_start, dst_start, len, pos0), ...] of one request under position re-use."""
+    spans = (ape_span_t * max(len(request.ctx), 1))(*[ape_span_t(int(s), int(l)) for s, l in request.ctx])
+    rq = ape_request_t(int(request.q_start), int(request.q_len), ape_span_t(*map(int, request.prefix)), spans,
+                       len(request.ctx), ape_span_t(*map(int, request.query_kv)), int(request.query_kv_capacity))
+    cap = len(request.ctx) + 2
+    runs = (ape_rope_run_t * cap)()
+    n = C.c_int32(0)
+    _check(load().ape_rope_runs_for_request(C.byref(rq), int(src_start), runs, cap, C.byref(n)), "ape_rope_runs_for_request")
+    return [(r.src_start, r.dst_start, r.len, r.pos0) for r in runs[: n.value]]
+
+
+class RopePlan:
+    """ape_rope_plan / ape_rope_write / ape_plan_destroy."""
+
+    def __init__(self, handle: "Handle", d: int, theta: float, runs: Sequence):
+        arr = (ape_rope_run_t * max(len(runs), 1))(*[ape_rope_run_t(*map(int, r)) for r in runs])
+        self._handle, self._p = handle, C.c_void_p()
+        _check(load().ape_rope_plan(handle._h, int(d), float(theta), arr, len(runs), C.byref(self._p)), "ape_rope_plan")
+
+    def write(self, src: torch.Tensor, dst: torch.Tensor, rotate: bool, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """ape_rope_write: src, dst bf16 [rows, heads, d] on the plan's device."""
+        st = stream if stream is not None else torch.cuda.current_stream(src.device)
+        sr, dr = _rows(src), _rows(dst)
+        _check(load().ape_rope_write(self._p, C.byref(sr), C.byref(dr), int(src.shape[1]), 1 if rotate else 0,
+                                     C.c_void_p(st.cuda_stream)), "ape_rope_write")
+
+    def close(self) -> None:
+        if self._p:
+            load().ape_plan_destroy(self._p)
+            self._p = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 class Plan:
