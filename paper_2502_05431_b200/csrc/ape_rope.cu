@@ -33,7 +33,7 @@ ape_rope_kernel(const RopeParams p)
 {
     constexpr int kHalf = D / 2;               // pairs per head
     constexpr int kVec = D / 16;               // 16-byte vectors per half head
-    __shared__ float2 table[2][kRopeChunkTokens][kHalf];       // (cos, sin) of the chunk's tokens, double-buffered
+    __shared__ __align__(16) float2 table[2][kRopeChunkTokens][kHalf];       // (cos, sin) of the chunk's tokens, double-buffered
 
     const int tid = threadIdx.x;
     // kRopeThreads is a multiple of kHalf: a thread always fills the same pair index of the table
@@ -61,7 +61,7 @@ ape_rope_kernel(const RopeParams p)
             __syncthreads();
         }
         const int n_items = ch.n_tok * p.n_heads * kVec;
-        #pragma unroll 2
+        #pragma unroll 4
         for (int it = tid; it < n_items; it += kRopeThreads) {
             const int v = it % kVec;
             const int h = (it / kVec) % p.n_heads;
@@ -79,13 +79,14 @@ ape_rope_kernel(const RopeParams p)
             }
             const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
             uint32_t lo[4], hi[4];
-            const float2* tb = &table[buf][t][v * 8];
+            // the thread's eight (cos, sin) pairs are 64 contiguous bytes: four 16-byte reads, free of bank conflicts
+            const float4* tb = reinterpret_cast<const float4*>(&table[buf][t][v * 8]);
             #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const float2 cs0 = tb[2 * j], cs1 = tb[2 * j + 1];
+                const float4 cs = tb[j];                           // (cos, sin) of pair 2j and of pair 2j + 1
                 const float a0 = bf16_lo(aw[j]), a1 = bf16_hi(aw[j]), b0 = bf16_lo(bw[j]), b1 = bf16_hi(bw[j]);
-                lo[j] = pack_rn(fmaf(a0, cs0.x, -b0 * cs0.y), fmaf(a1, cs1.x, -b1 * cs1.y));
-                hi[j] = pack_rn(fmaf(b0, cs0.x, a0 * cs0.y), fmaf(b1, cs1.x, a1 * cs1.y));
+                lo[j] = pack_rn(fmaf(a0, cs.x, -b0 * cs.y), fmaf(a1, cs.z, -b1 * cs.w));
+                hi[j] = pack_rn(fmaf(b0, cs.x, a0 * cs.y), fmaf(b1, cs.z, a1 * cs.w));
             }
             *reinterpret_cast<uint4*>(dst) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             *reinterpret_cast<uint4*>(dst + kHalf) = make_uint4(hi[0], hi[1], hi[2], hi[3]);

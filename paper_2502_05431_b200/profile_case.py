@@ -21,7 +21,7 @@ from . import libape, workloads as wl
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["prefill", "decode", "encode", "rag"])
+    ap.add_argument("case", choices=["prefill", "decode", "encode", "rag", "rope"])
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--n-ctx", type=int, default=250)
     args = ap.parse_args()
@@ -47,6 +47,22 @@ def main():
         ws = plan.alloc_workspace()
         run = lambda: plan.attend(b.T, b.S, ws)
         work = {"bytes": 4 * (64 + args.n_ctx * 256 + 257) * 4.0 * H_kv * d}
+    elif args.case == "rope":
+        # the step in front of the pre-caching attention: n_ctx contexts of 256 tokens behind a 64-token prefix;
+        # K rotated (H_kv heads), V copied, Q rotated (H_q heads), all written at their cache rows
+        n_tok = 64 + args.n_ctx * 256
+        runs = [(0, 0, 64, 0)] + [(64 + i * 256, 64 + i * 256, 256, 64) for i in range(args.n_ctx)]
+        g = torch.Generator(device=dev).manual_seed(1)
+        k_raw = torch.randn(n_tok, H_kv, d, generator=g, device=dev).to(torch.bfloat16)
+        v_raw = torch.randn(n_tok, H_kv, d, generator=g, device=dev).to(torch.bfloat16)
+        q_raw = torch.randn(n_tok, H_q, d, generator=g, device=dev).to(torch.bfloat16)
+        k_pool, v_pool, q_enc = torch.empty_like(k_raw), torch.empty_like(v_raw), torch.empty_like(q_raw)
+        plan = libape.RopePlan(h, d, 500000.0, runs)
+        def run():
+            plan.write(k_raw, k_pool, True)
+            plan.write(v_raw, v_pool, False)
+            plan.write(q_raw, q_enc, True)
+        work = {"bytes": 2.0 * 2 * n_tok * d * (2 * H_kv + H_q)}
     else:
         b = wl.config4(n_ctx=args.n_ctx, with_encode_q=(args.case == "encode"), device=dev)
         if args.case == "prefill":
