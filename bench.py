@@ -2,6 +2,8 @@
 """Benchmark of the APE attention hot path at 128K context on B200.
 
 One step = one pass of the whole path over one batch of synthetic input:
+  rope     rotary embedding with position re-use of the raw K, Q (rotated) and V (copied) of the prefix and the 500
+           contexts, written to their cache rows (HBM bound),
   encode   500 contexts x 256 tokens against a 64-token shared prefix (block-diagonal attention),
   prefill  256 query rows over prefix 64 + 128,000 cached context tokens + causal self (many-shot 128K case),
   decode   one new token for each of 16 requests over prefix 64 + 128,000 + 257 cached tokens.
@@ -210,6 +212,13 @@ def main():
     e_out = torch.zeros_like(pb.q_enc)
     plan_e = h.encode_plan(H_q=H_Q, H_kv=H_KV, d=D, k_pool=pb.k_pool, v_pool=pb.v_pool, q=pb.q_enc, out=e_out,
                            prefix=rq.prefix, ctx=rq.ctx)
+    # raw (un-rotated) K, V, Q of the prefix and the contexts, packed in request order; the rope leg writes them into the
+    # pool rows that the encode leg reads (a rotation keeps the N(0,1) statistics of the synthetic data)
+    runs = libape.rope_runs_for_request(rq, 0)[:-1]
+    n_raw = sum(r[2] for r in runs)
+    k_raw, v_raw, q_raw = pb.k_pool[:n_raw].clone(), pb.v_pool[:n_raw].clone(), pb.q_enc[:n_raw].clone()
+    plan_r = libape.RopePlan(h, D, 500000.0, runs)
+    by_rope = 2.0 * 2 * n_raw * D * (2 * H_KV + H_Q)
     d_q = db.extra["q_steps"][0].contiguous()
     d_out = torch.zeros_like(d_q)
     plan_d = h.attend_plan(H_q=H_Q, H_kv=H_KV, d=D, k_pool=db.k_pool, v_pool=db.v_pool, q=d_q, out=d_out,
@@ -222,6 +231,10 @@ def main():
     fl_decode = 4.0 * D * H_Q * DEC_REQ * (L_P + N_CTX * L_CTX + DEC_LK)
 
     def step(ev=None):
+        if ev: ev[4].record()
+        plan_r.write(k_raw, pb.k_pool, True)
+        plan_r.write(v_raw, pb.v_pool, False)
+        plan_r.write(q_raw, pb.q_enc, True)
         if ev: ev[0].record()
         plan_e.encode_contexts()
         if ev: ev[1].record()
@@ -236,7 +249,7 @@ def main():
     assert h.get_status() == 0, "a kernel reported a timed-out wait"
 
     sampler = ClockSampler(local_rank)
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
     if dist:
         td.barrier()
     torch.cuda.synchronize()
@@ -254,8 +267,9 @@ def main():
     t_enc = sum(e[0].elapsed_time(e[1]) for e in events) / args.steps
     t_pre = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
     t_dec = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
-    t_step = events[0][0].elapsed_time(events[-1][3]) / args.steps
-    t_enc, t_pre, t_dec, t_step = dist_util.max_over_ranks([t_enc, t_pre, t_dec, t_step], dev)
+    t_rope = sum(e[4].elapsed_time(e[0]) for e in events) / args.steps
+    t_step = events[0][4].elapsed_time(events[-1][3]) / args.steps
+    t_enc, t_pre, t_dec, t_step, t_rope = dist_util.max_over_ranks([t_enc, t_pre, t_dec, t_step, t_rope], dev)
 
     # ---- end to end through the host-buffer entry point (prefill half of the metric) ---------------------------------
     e2e = None
@@ -290,20 +304,24 @@ def main():
     roof_dec = {"bound": "hbm", "kernel": "ape_decode_kernel<128> (+ merge)", "achieved": gbs_decode, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": gbs_decode / peaks["hbm_gbs"], "traffic": ncu_traffic("decode"), "peak_source": f"{peaks['source']} copy",
                 "frac_of_nominal_8000": gbs_decode / 8000.0}
+    gbs_rope = by_rope / (t_rope * 1e-3) / 1e9
+    roof_rope = {"bound": "hbm", "kernel": "ape_rope_kernel<128> x3 (K, V, Q)", "achieved": gbs_rope, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                 "frac": gbs_rope / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peaks['source']} copy"}
     cpu = None if args.no_cpu_baseline else cpu_oracle_sample()
     line = {
         "metric": METRIC, "value": world * tf_prefill, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": t_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "cfg4_manyshot_128k prefill (value) + cfg5 decode x16 + encode 500x256, Llama-3-8B head shape",
+        "config": {"workload": "cfg4_manyshot_128k prefill (value) + cfg5 decode x16 + rope/encode 500x256, Llama-3-8B head shape",
                    "H_q": H_Q, "H_kv": H_KV, "d": D, "prefix": L_P, "contexts": f"{N_CTX}x{L_CTX}", "query_rows": L_Q,
                    "decode_batch": DEC_REQ, "T": pb.T, "S": pb.S, "l2": "inputs larger than L2 (0.53 GB / 8.4 GB KV per pass)",
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
         "prefill": {"ms": t_pre, "tflops": tf_prefill, "flops": fl_prefill},
         "decode": {"ms_per_step": t_dec, "value": world * gbs_decode, "unit": "GB/s", "bytes": by_decode, "tflops": fl_decode / (t_dec * 1e-3) / 1e12,
                    "roofline": roof_dec},
+        "rope": {"ms": t_rope, "value": world * gbs_rope, "unit": "GB/s", "bytes": by_rope, "roofline": roof_rope},
         "encode": {"ms": t_enc, "tflops": tf_encode, "flops": fl_encode, "frac_of_sustained_peak": tf_encode / peaks["tf_sustained"]},
         "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
-        "gpu_launches": args.steps * (plan_e.last_launches() + plan_p.last_launches() + plan_d.last_launches()),
+        "gpu_launches": args.steps * (3 + plan_e.last_launches() + plan_p.last_launches() + plan_d.last_launches()),
         "wall_s_timed_region": t_wall,
     }
     print(json.dumps(line))

@@ -53,7 +53,7 @@ ape_rope_kernel(const RopeParams p)
                 double r = fma(-k, k2PiHi, ang);
                 r = fma(-k, k2PiLo, r);
                 float sn, cs;
-                sincosf(static_cast<float>(r), &sn, &cs);
+                __sincosf(static_cast<float>(r), &sn, &cs);       // |r| <= pi: the fast form is good to a few 1e-7 there
                 table[buf][t][my_i] = make_float2(cs, sn);
             }
             // One barrier per chunk is enough with two tables: a thread can only reach the fill of this buffer's next
