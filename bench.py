@@ -57,8 +57,9 @@ def decode_bytes(n_req: int, tokens_per_req: int) -> float:
 # cached tokens).  Valid only for the kernel sources the counters were taken with: the figure is dropped (null) as
 # soon as the hash of those sources changes.
 NCU_TRAFFIC = {
-    "prefill": {"bytes": 2 * (267.07e6 + 10.48e6), "sources": ["ape_attn.cu", "ape_tcgen05.cuh", "ape_common.cuh"], "sha": "9d2800857a8865cb"},
-    "decode": {"bytes": (1.05515e9 + 4.08e6) * (8409907200.0 / 1053835264.0), "sources": ["ape_decode.cu", "ape_common.cuh"], "sha": "40414ccd4470df96"},
+    "prefill": {"bytes": 2 * (267.08e6 + 10.62e6), "sources": ["ape_attn.cu", "ape_tcgen05.cuh", "ape_common.cuh"], "sha": "cded79e3ef596482"},
+    "decode": {"bytes": (1.05518e9 + 3.89e6) * (8409907200.0 / 1053835264.0), "sources": ["ape_decode.cu", "ape_common.cuh"], "sha": "4c5dfbc56ad11182"},
+    "rope": {"bytes": 2 * ((131.30e6 + 87.13e6) + (131.30e6 + 82.04e6) + (524.91e6 + 479.47e6)), "sources": ["ape_rope.cu"], "sha": "f5898872292cd437"},
 }
 
 
@@ -306,7 +307,7 @@ def main():
                 "frac_of_nominal_8000": gbs_decode / 8000.0}
     gbs_rope = by_rope / (t_rope * 1e-3) / 1e9
     roof_rope = {"bound": "hbm", "kernel": "ape_rope_kernel<128> x3 (K, V, Q)", "achieved": gbs_rope, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                 "frac": gbs_rope / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peaks['source']} copy"}
+                 "frac": gbs_rope / peaks["hbm_gbs"], "traffic": ncu_traffic("rope"), "peak_source": f"{peaks['source']} copy"}
     cpu = None if args.no_cpu_baseline else cpu_oracle_sample()
     line = {
         "metric": METRIC, "value": world * tf_prefill, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
