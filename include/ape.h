@@ -111,6 +111,20 @@ int ape_attend_plan_per_context(ape_handle_t handle, const ape_shape_t *shape, c
                                 const ape_request_t *requests, int32_t n_req, ape_mode_t mode, ape_plan_t *plan);
 
 /*
+ * Decode for a batch of requests that attend to the SAME cached contexts (the serving case the paper's cache argument
+ * describes: many queries over one set of pre-encoded documents or shots; section "Parallel Encoding", pre-caching).
+ * Every request has q_len 1, its row of Q directly follows the previous request's (q_start = requests[0].q_start + r),
+ * and the context tokens of all requests are the same set (any split into contexts, any order); prefixes and query
+ * segments are per request.  The context K/V is then read ONCE for the whole batch: the context pass runs on the tensor
+ * cores with the batch's query rows as one block of rows, the rest (prefix + the request's own growing query segment)
+ * runs per request, and one merge applies Eq. 5 per request.  Launch with ape_attend (T, S, kv_extra as for APE_DECODE).
+ * APE_ERR_INVALID_ARG if the requests do not share their contexts or their rows are not consecutive.
+ */
+int ape_attend_plan_shared(ape_handle_t handle, const ape_shape_t *shape, const ape_kv_pool_t *pool,
+                           const ape_rows_t *q, const ape_rows_t *out, float *lse,
+                           const ape_request_t *requests, int32_t n_req, ape_plan_t *plan);
+
+/*
  * Plan the block-diagonal encoding of n_ctx contexts against one shared prefix.  `q` and `out` are aligned
  * with the pool: row t belongs to pool token t (only rows inside the context spans are read / written).
  * `lse` (nullable, fp32 [pool rows, H_q]) receives each row's log-sum-exp.

@@ -14,7 +14,7 @@ using namespace ape;
 
 namespace {
 
-enum PlanKind { PLAN_PREFILL = 0, PLAN_DECODE = 1, PLAN_ENCODE = 2, PLAN_ROPE = 3 };
+enum PlanKind { PLAN_PREFILL = 0, PLAN_DECODE = 1, PLAN_ENCODE = 2, PLAN_ROPE = 3, PLAN_SHARED = 4 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -55,6 +55,9 @@ struct ape_plan_s {
     bool o_via_tma = false;         // encode plans: tm_o describes the output rows
     int32_t last_launches = 0;
     bool per_context = false;        // merge form: Eq. 5 (false) or Eq. 11-12 (true)
+    // shared-context decode plans: the context pass of all requests (tensor-core kernel) and the per-request rest (decode kernel)
+    ape_plan_s* child_ctx = nullptr;
+    ape_plan_s* child_oth = nullptr;
     // rotary-embedding plans
     RopeChunk* d_rope_chunks = nullptr;
     int n_rope_chunks = 0;
@@ -194,7 +197,7 @@ void assign_stream(const std::vector<Run>& runs, int n_bins, int slot_mult, Host
             // bookkeeping for the merge: every live sibling's group record learns about this partial
             for (int s = 0; s < r.n_sib; ++s) {
                 DevMerge& g = m.merge[r.merge0 + s];
-                g.slot_stride = slot_mult;
+                g.slot_stride = slot_mult; g.ctx_stride = slot_mult;
                 if (r.seg == SEG_CTX) { if (g.ctx_n == 0) g.ctx_slot0 = it.slot + s; g.ctx_n++; }
                 else { if (g.oth_n == 0) g.oth_slot0 = it.slot + s; g.oth_n++; }
             }
@@ -287,6 +290,8 @@ int ape_destroy(ape_handle_t h) {
 
 int ape_plan_destroy(ape_plan_t p) {
     if (!p) return APE_ERR_INVALID_ARG;
+    if (p->child_ctx) ape_plan_destroy(p->child_ctx);
+    if (p->child_oth) ape_plan_destroy(p->child_oth);
     if (p->d_blob) { cudaSetDevice(p->h->device); cudaFree(p->d_blob); }
     delete p;
     return APE_OK;
@@ -423,6 +428,141 @@ int ape_attend_plan_per_context(ape_handle_t h, const ape_shape_t* shape, const 
                                 ape_plan_t* plan_out)
 {
     return attend_plan_impl(h, shape, pool, q, out, lse, reqs, n_req, mode, true, plan_out);
+}
+
+int ape_attend_plan_shared(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
+                           const ape_rows_t* out, float* lse, const ape_request_t* reqs, int32_t n_req, ape_plan_t* plan_out)
+{
+    if (!h || !plan_out) return APE_ERR_INVALID_ARG;
+    *plan_out = nullptr;
+    int G = 1; float c = 0.f;
+    int rc = check_shape(shape, &G, &c);              if (rc) return rc;
+    rc = check_pool(pool, shape);                     if (rc) return rc;
+    rc = check_rows(q, shape);                        if (rc) return rc;
+    rc = check_rows(out, shape);                      if (rc) return rc;
+    if (!reqs || n_req <= 0 || out->n_rows < q->n_rows) return APE_ERR_INVALID_ARG;
+    int64_t max_extra = INT64_MAX;
+    std::vector<ape_span_t> shared_ctx;
+    for (int r = 0; r < n_req; ++r) {
+        const ape_request_t& rq = reqs[r];
+        if (rq.q_len != 1 || rq.q_start != reqs[0].q_start + r || rq.q_start < 0 || rq.q_start + 1 > q->n_rows) return APE_ERR_INVALID_ARG;
+        if (rq.n_ctx < 0 || (rq.n_ctx > 0 && !rq.ctx)) return APE_ERR_INVALID_ARG;
+        if (!span_ok(rq.prefix, pool->n_tokens) || !span_ok(rq.query_kv, pool->n_tokens)) return APE_ERR_INVALID_ARG;
+        for (int i = 0; i < rq.n_ctx; ++i) if (!span_ok(rq.ctx[i], pool->n_tokens)) return APE_ERR_INVALID_ARG;
+        if (rq.query_kv.len < 1) return APE_ERR_INVALID_ARG;
+        if (rq.query_kv_capacity < rq.query_kv.len || rq.query_kv.start + rq.query_kv_capacity > pool->n_tokens) return APE_ERR_INVALID_ARG;
+        max_extra = std::min(max_extra, rq.query_kv_capacity - rq.query_kv.len);
+        // the same context tokens for every request (Eq. 5 does not care how they are cut into contexts, or in which order)
+        std::vector<ape_span_t> mine = fuse_spans(rq.ctx, rq.n_ctx);
+        if (r == 0) shared_ctx = mine;
+        else {
+            if (mine.size() != shared_ctx.size()) return APE_ERR_INVALID_ARG;
+            for (size_t i = 0; i < mine.size(); ++i)
+                if (mine[i].start != shared_ctx[i].start || mine[i].len != shared_ctx[i].len) return APE_ERR_INVALID_ARG;
+        }
+    }
+    rc = set_device(h); if (rc) return rc;
+    const int D = shape->head_dim, H_kv = shape->n_kv_heads;
+
+    auto new_plan = [&](PlanKind kind) {
+        ape_plan_t p = new (std::nothrow) ape_plan_s();
+        if (p) { p->h = h; p->kind = kind; p->shape = *shape; p->c = c; p->G = G; p->pool = *pool; p->q = *q; p->out = *out; p->lse = lse; }
+        return p;
+    };
+    ape_plan_t p = new_plan(PLAN_SHARED);
+    if (!p) return APE_ERR_NOMEM;
+    p->max_kv_extra = max_extra;
+    p->child_ctx = new_plan(PLAN_PREFILL);
+    p->child_oth = new_plan(PLAN_DECODE);
+    if (!p->child_ctx || !p->child_oth) { ape_plan_destroy(p); return APE_ERR_NOMEM; }
+    try {
+        // ---- context pass: the requests' query rows are the "tokens" of one row-block sequence ------------------------
+        ape_plan_t a = p->child_ctx;
+        HostMeta ma;
+        std::vector<Run> runs_a;
+        const int TB = kAttnRows / G;
+        const int RB = (n_req + TB - 1) / TB;
+        a->n_sib = std::min(4, RB);
+        const int n_groups = std::max(1, h->n_sm / a->n_sib);
+        ma.reqs.push_back(DevReq{static_cast<int32_t>(reqs[0].q_start), n_req, n_req, 0});
+        const int t0 = 0;
+        for (const auto& sp : shared_ctx) add_span_tiles(ma.tiles, sp.start, sp.len, kAttnTileN, 0, 0);
+        const int t1 = static_cast<int>(ma.tiles.size());
+        for (int hh = 0; hh < H_kv; ++hh)
+            for (int rb0 = 0; rb0 < RB; rb0 += a->n_sib) {
+                const int live = std::min(a->n_sib, RB - rb0);
+                const int mi = static_cast<int>(ma.merge.size());
+                for (int sb = 0; sb < live; ++sb) ma.merge.push_back(DevMerge{0, hh, rb0 + sb, 0, 0, 0, 0, 1});
+                if (t1 > t0) runs_a.push_back(Run{0, hh, rb0, live, SEG_CTX, t0, t1, mi});
+            }
+        assign_stream(runs_a, n_groups, a->n_sib, ma);
+        a->n_cta = n_groups * a->n_sib;
+        a->n_slots = static_cast<int>(ma.items.size()) * a->n_sib;
+        a->smem_bytes = attn_smem_bytes(D, 1);
+        rc = make_map(h, &a->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, kAttnTileN);
+        if (!rc) rc = make_map(h, &a->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, kAttnTileN);
+        if (!rc) rc = make_map(h, &a->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
+        if (!rc && attn_set_smem_attr(D, 1, a->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+        if (!rc) { finish_items(ma); rc = upload(a, ma); }
+
+        // ---- the rest, per request: prefix + the request's own (growing) query segment ------------------------------
+        ape_plan_t b = p->child_oth;
+        HostMeta mb;
+        std::vector<Run> runs_b;
+        for (int r = 0; r < n_req && !rc; ++r) {
+            const ape_request_t& rq = reqs[r];
+            mb.reqs.push_back(DevReq{static_cast<int32_t>(rq.q_start), 1, static_cast<int32_t>(rq.query_kv.len), 0});
+            const int o0 = static_cast<int>(mb.tiles.size());
+            add_span_tiles(mb.tiles, rq.prefix.start, rq.prefix.len, kDecodeTile, 0, 0);
+            add_span_tiles(mb.tiles, rq.query_kv.start, rq.query_kv.len, kDecodeTile, TILE_GROWS, rq.query_kv_capacity);
+            const int o1 = static_cast<int>(mb.tiles.size());
+            for (int hh = 0; hh < H_kv; ++hh) {
+                const int mi = static_cast<int>(mb.merge.size());
+                mb.merge.push_back(DevMerge{r, hh, 0, 0, 0, 0, 0, 1});
+                runs_b.push_back(Run{r, hh, 0, 1, SEG_OTHER, o0, o1, mi});
+            }
+        }
+        if (!rc) {
+            b->n_sib = 1; b->n_cta = h->n_sm;
+            assign_stream(runs_b, b->n_cta, 1, mb);
+            b->n_slots = static_cast<int>(mb.items.size());
+            b->n_stages = decode_pick_stages(D, G, h->smem_optin - 2048);
+            if (b->n_stages < 2) rc = APE_ERR_SHAPE;
+        }
+        if (!rc) {
+            b->smem_bytes = decode_smem_bytes(D, G, b->n_stages);
+            rc = make_map(h, &b->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, kDecodeTile);
+            if (!rc) rc = make_map(h, &b->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, kDecodeTile);
+            if (!rc && decode_set_smem_attr(D, b->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+            if (!rc) { finish_items(mb); rc = upload(b, mb); }
+        }
+
+        // ---- merge records of the whole plan: context partials from the first pass, the rest from the second -----------
+        if (!rc) {
+            HostMeta mp;
+            mp.reqs = mb.reqs;
+            for (int r = 0; r < n_req; ++r)
+                for (int hh = 0; hh < H_kv; ++hh) {
+                    const DevMerge& ga = ma.merge[static_cast<size_t>(hh) * RB + r / TB];
+                    const DevMerge& gb = mb.merge[static_cast<size_t>(r) * H_kv + hh];
+                    DevMerge g{r, hh, 0, ga.ctx_slot0, ga.ctx_n, gb.oth_slot0, gb.oth_n, std::max(1, gb.slot_stride)};
+                    g.ctx_row_off = (r % TB) * G;
+                    g.ctx_stride = ga.ctx_stride;
+                    mp.merge.push_back(g);
+                }
+            rc = upload(p, mp);
+            auto rnd = [](size_t x) { return (x + 255) & ~size_t(255); };
+            const size_t rows_a = static_cast<size_t>(a->n_slots) * kAttnRows, rows_b = static_cast<size_t>(b->n_slots) * G;
+            a->ws_bytes = rnd(rows_a * D * 4) + rnd(rows_a * 2 * 4);
+            b->ws_bytes = rnd(rows_b * D * 4) + rnd(rows_b * 2 * 4);
+            p->ws_bytes = a->ws_bytes + b->ws_bytes;
+        }
+    } catch (const std::bad_alloc&) {
+        rc = APE_ERR_NOMEM;
+    }
+    if (rc) { ape_plan_destroy(p); return rc; }
+    *plan_out = p;
+    return APE_OK;
 }
 
 int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
@@ -600,7 +740,7 @@ int ape_plan_last_launches(ape_plan_t p, int32_t* n) {
 
 int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace, size_t ws_bytes, void* stream_v) {
     if (!p) return APE_ERR_INVALID_ARG;
-    if (p->kind != PLAN_PREFILL && p->kind != PLAN_DECODE) return APE_ERR_MODE;
+    if (p->kind != PLAN_PREFILL && p->kind != PLAN_DECODE && p->kind != PLAN_SHARED) return APE_ERR_MODE;
     if (!(T > 0.f) || !(S > 0.f) || !std::isfinite(T) || !std::isfinite(S)) return APE_ERR_RANGE;
     if (kv_extra < 0 || kv_extra > p->max_kv_extra) return APE_ERR_RANGE;
     if (p->ws_bytes > 0 && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || ws_bytes < p->ws_bytes)) return APE_ERR_WORKSPACE;
@@ -608,6 +748,43 @@ int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const int D = p->shape.head_dim, G = p->G;
     constexpr float kLog2e = 1.4426950408889634f;
+    if (p->kind == PLAN_SHARED) {
+        // context pass of all requests at once, the per-request rest, then one merge that reads both sets of partials
+        ape_plan_t a = p->child_ctx, b = p->child_oth;
+        auto rnd = [](size_t x) { return (x + 255) & ~size_t(255); };
+        const size_t rows_a = static_cast<size_t>(a->n_slots) * kAttnRows, rows_b = static_cast<size_t>(b->n_slots) * G;
+        uint8_t* base = static_cast<uint8_t*>(workspace);
+        float* a_o = reinterpret_cast<float*>(base);
+        float* a_ml = reinterpret_cast<float*>(base + rnd(rows_a * D * 4));
+        float* b_o = reinterpret_cast<float*>(base + a->ws_bytes);
+        float* b_ml = reinterpret_cast<float*>(base + a->ws_bytes + rnd(rows_b * D * 4));
+        p->last_launches = 0;
+        if (a->n_items > 0) {
+            AttnParams ap;
+            ap.tiles = a->d_tiles; ap.items = a->d_items; ap.cta_item_begin = a->d_cta_begin; ap.reqs = a->d_reqs;
+            ap.out = rows_desc(p->out); ap.lse_out = nullptr; ap.ws_o = a_o; ap.ws_ml = a_ml;
+            ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c / T * kLog2e;
+            ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = a->n_sib; ap.n_q_bufs = 1; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
+            ap.o_via_tma = 0;
+            if (launch_attn(D, a->tm_q, a->tm_k, a->tm_v, a->tm_q, ap, a->n_cta, a->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
+            p->last_launches++;
+        }
+        DecodeParams dp;
+        dp.tiles = b->d_tiles; dp.items = b->d_items; dp.cta_item_begin = b->d_cta_begin; dp.reqs = b->d_reqs;
+        dp.q = rows_desc(p->q); dp.ws_o = b_o; dp.ws_ml = b_ml;
+        dp.scale_oth_log2 = p->c * kLog2e; dp.scale_ctx_log2 = p->c / T * kLog2e;
+        dp.kv_extra = static_cast<int32_t>(kv_extra); dp.G = G; dp.n_stages = b->n_stages; dp.status = p->h->d_status;
+        if (launch_decode(D, b->tm_k, b->tm_v, dp, b->n_cta, b->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
+        p->last_launches++;
+        MergeParams mp;
+        mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.items = nullptr; mp.per_context = 0; mp.n_groups = p->n_merge;
+        mp.rows_per_slot = G; mp.tokens_per_block = 1; mp.ws_o = b_o; mp.ws_ml = b_ml;
+        mp.ws_o_ctx = a_o; mp.ws_ml_ctx = a_ml; mp.rows_per_slot_ctx = kAttnRows;
+        mp.out = rows_desc(p->out); mp.lse_out = p->lse; mp.S = S; mp.G = G; mp.H_q = p->shape.n_q_heads; mp.D = D;
+        if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;
+        p->last_launches++;
+        return APE_OK;
+    }
     const int rows_per_slot = (p->kind == PLAN_DECODE) ? G : kAttnRows;
     const size_t rows = static_cast<size_t>(p->n_slots) * rows_per_slot;
     float* ws_o = static_cast<float*>(workspace);
@@ -635,6 +812,7 @@ int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace
     MergeParams mp;
     mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.items = p->d_items; mp.per_context = p->per_context ? 1 : 0; mp.n_groups = p->n_merge; mp.rows_per_slot = rows_per_slot;
     mp.tokens_per_block = rows_per_slot / G; mp.ws_o = ws_o; mp.ws_ml = ws_ml; mp.out = rows_desc(p->out); mp.lse_out = p->lse;
+    mp.ws_o_ctx = ws_o; mp.ws_ml_ctx = ws_ml; mp.rows_per_slot_ctx = rows_per_slot;
     mp.S = S; mp.G = G; mp.H_q = p->shape.n_q_heads; mp.D = D;
     if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;
     p->last_launches++;
@@ -870,6 +1048,7 @@ int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, cons
     MergeParams mp;
     mp.groups = reinterpret_cast<const DevMerge*>(base + o_merge); mp.reqs = dp.reqs; mp.items = dp.items; mp.per_context = 0; mp.n_groups = static_cast<int32_t>(m.merge.size());
     mp.rows_per_slot = G; mp.tokens_per_block = 1; mp.ws_o = ws_o; mp.ws_ml = ws_ml; mp.out = rows_desc(*out); mp.lse_out = lse;
+    mp.ws_o_ctx = ws_o; mp.ws_ml_ctx = ws_ml; mp.rows_per_slot_ctx = G;
     mp.S = S; mp.G = G; mp.H_q = shape->n_q_heads; mp.D = D;
     if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;
     if (device_status != nullptr) {

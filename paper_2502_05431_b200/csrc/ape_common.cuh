@@ -58,7 +58,10 @@ struct DevMerge {
     int32_t ctx_n;
     int32_t oth_slot0;
     int32_t oth_n;
-    int32_t slot_stride;
+    int32_t slot_stride; // between consecutive non-context partials (and context partials of ordinary plans)
+    int32_t ctx_row_off; // added to the row when a context partial is read: shared-context plans keep the context
+                         // partials of many requests in one slot, one group of rows per request
+    int32_t ctx_stride;  // between consecutive context partials
 };
 
 struct RowsDesc {        // Q or O rows: element (r, h, e) at data[r*token_stride + h*head_stride + e]

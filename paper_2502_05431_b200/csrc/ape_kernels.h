@@ -69,6 +69,10 @@ struct MergeParams {
     int32_t tokens_per_block;        // query tokens per row block: rows_per_slot / G
     const float* ws_o;
     const float* ws_ml;
+    // context partials; ordinary plans keep them in the same workspace with the same geometry as the others
+    const float* ws_o_ctx;
+    const float* ws_ml_ctx;
+    int32_t rows_per_slot_ctx;
     RowsDesc out;
     float* lse_out;                  // nullable, [rows, H_q]
     float S;

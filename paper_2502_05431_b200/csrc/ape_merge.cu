@@ -110,7 +110,8 @@ __global__ void __launch_bounds__(256) ape_merge_kernel(const MergeParams p)
     if (p.per_context) {
         combine_per_context<VEC>(p, g, row, lane, lse_c, Lc, ac);      // Lc: the normaliser of ac
     } else {
-        combine_segment<VEC>(p.ws_o, p.ws_ml, g.ctx_slot0, g.ctx_n, g.slot_stride, p.rows_per_slot, row, p.D, lane, Mc, Lc, ac);
+        combine_segment<VEC>(p.ws_o_ctx, p.ws_ml_ctx, g.ctx_slot0, g.ctx_n, g.ctx_stride, p.rows_per_slot_ctx, row + g.ctx_row_off,
+                             p.D, lane, Mc, Lc, ac);
         // base-2 log-sum-exp of the context segment, multiplied by S (Eq. 5: Z_C^S)
         lse_c = (Lc > 0.f) ? p.S * (Mc + fast_log2(Lc)) : -INFINITY;
     }

@@ -20,7 +20,7 @@ APE_PREFILL, APE_DECODE = 0, 1
 EXPORTS = ["ape_create", "ape_destroy", "ape_attend_plan", "ape_encode_plan", "ape_plan_workspace_bytes",
            "ape_plan_destroy", "ape_attend", "ape_encode_contexts", "ape_attend_host", "ape_plan_last_launches",
            "ape_get_status", "ape_status_string", "ape_decode_noalloc", "ape_attend_plan_per_context",
-           "ape_rope_runs_for_request", "ape_rope_plan", "ape_rope_write"]
+           "ape_rope_runs_for_request", "ape_rope_plan", "ape_rope_write", "ape_attend_plan_shared"]
 
 
 class ApeError(RuntimeError):
@@ -71,6 +71,7 @@ def load() -> C.CDLL:
         lib.ape_attend_plan.argtypes = [vp, C.POINTER(ape_shape_t), C.POINTER(ape_kv_pool_t), C.POINTER(ape_rows_t),
                                         C.POINTER(ape_rows_t), vp, C.POINTER(ape_request_t), C.c_int32, C.c_int, C.POINTER(vp)]
         lib.ape_attend_plan_per_context.argtypes = lib.ape_attend_plan.argtypes
+        lib.ape_attend_plan_shared.argtypes = lib.ape_attend_plan.argtypes[:7] + lib.ape_attend_plan.argtypes[8:]
         lib.ape_encode_plan.argtypes = [vp, C.POINTER(ape_shape_t), C.POINTER(ape_kv_pool_t), C.POINTER(ape_rows_t),
                                         C.POINTER(ape_rows_t), vp, C.POINTER(ape_span_t), C.POINTER(ape_span_t), C.c_int32,
                                         C.POINTER(vp)]
@@ -178,8 +179,10 @@ class Handle:
 
     def attend_plan(self, *, H_q: int, H_kv: int, d: int, k_pool: torch.Tensor, v_pool: torch.Tensor,
                     q: torch.Tensor, out: torch.Tensor, requests: Sequence, mode: int,
-                    lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0, per_context: bool = False) -> "Plan":
-        """ape_attend_plan (or ape_attend_plan_per_context: S on every context's own LSE, Eq. 11-12).  `requests`: objects with q_start, q_len, prefix, ctx, query_kv, query_kv_capacity
+                    lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0, per_context: bool = False,
+                    shared: bool = False) -> "Plan":
+        """ape_attend_plan (or ape_attend_plan_per_context: S on every context's own LSE, Eq. 11-12; or, with shared=True,
+        ape_attend_plan_shared: a decode batch whose requests all attend to the same contexts).  `requests`: objects with q_start, q_len, prefix, ctx, query_kv, query_kv_capacity
         (spans are (start, len) pairs), e.g. paper_2502_05431_b200.workloads.Request."""
         shape = ape_shape_t(H_q, H_kv, d, softmax_scale)
         pool, qr, orows = _pool(k_pool, v_pool), _rows(q), _rows(out)
@@ -192,6 +195,11 @@ class Handle:
             arr[i] = ape_request_t(int(r.q_start), int(r.q_len), ape_span_t(*map(int, r.prefix)), spans, len(r.ctx),
                                    ape_span_t(*map(int, r.query_kv)), int(r.query_kv_capacity))
         p = C.c_void_p()
+        if shared:
+            _check(load().ape_attend_plan_shared(self._h, C.byref(shape), C.byref(pool), C.byref(qr), C.byref(orows),
+                                                 lse.data_ptr() if lse is not None else None, arr, n, C.byref(p)),
+                   "ape_attend_plan_shared")
+            return Plan(self, p, (q, out, k_pool, v_pool, lse))
         fn = load().ape_attend_plan_per_context if per_context else load().ape_attend_plan
         _check(fn(self._h, C.byref(shape), C.byref(pool), C.byref(qr), C.byref(orows),
                   lse.data_ptr() if lse is not None else None, arr, n, int(mode), C.byref(p)),

@@ -69,6 +69,18 @@ def _randn_bf16(gen: torch.Generator, shape, scale: Optional[torch.Tensor] = Non
     return x.to(torch.bfloat16)
 
 
+def share_contexts(b: Batch) -> Batch:
+    """The same tensors with every request pointed at request 0's contexts (each keeps its own prefix, query rows and
+    query segment): a batch of queries over one set of cached contexts.  The span tables of the requests list the shared
+    contexts in different (rotated) orders."""
+    ctx0 = list(b.requests[0].ctx)
+    reqs = []
+    for i, r in enumerate(b.requests):
+        k = i % max(len(ctx0), 1)
+        reqs.append(Request(r.q_start, r.q_len, r.prefix, ctx0[k:] + ctx0[:k], r.query_kv, r.query_kv_capacity))
+    return Batch(b.H_q, b.H_kv, b.d, b.q, b.k_pool, b.v_pool, reqs, b.T, b.S, b.q_enc, b.name + "+shared", dict(b.extra))
+
+
 def make_batch(*, H_q: int, H_kv: int, d: int, l_P: int, ctx_lens: Sequence[Sequence[int]], l_q: int,
                l_k: Optional[int] = None, capacity: Optional[int] = None, seed: int = 0,
                T: float = 1.0, S: float = 1.0, head_scale: bool = False, gap: int = 0,
