@@ -6,7 +6,8 @@ One step = one pass of the whole path over one batch of synthetic input:
            contexts, written to their cache rows (HBM bound),
   encode   500 contexts x 256 tokens against a 64-token shared prefix (block-diagonal attention),
   prefill  256 query rows over prefix 64 + 128,000 cached context tokens + causal self (many-shot 128K case),
-  decode   one new token for each of 16 requests over prefix 64 + 128,000 + 257 cached tokens.
+  decode   one new token for each of 16 requests over prefix 64 + 128,000 + 257 cached tokens,
+  shared   the same decode step when all 16 requests attend to one set of contexts (read once for the batch).
 The headline metric has two halves: `value` is the prefill half (TFLOP/s, tensor-core bound) and `decode`
 carries the decode half (GB/s, HBM bound).  Inputs are resident in HBM before the timed region and larger than
 L2 (KV 0.53 GB for prefill, 8.4 GB for decode), so no L2 flush is needed between iterations.
@@ -225,6 +226,12 @@ def main():
     plan_d = h.attend_plan(H_q=H_Q, H_kv=H_KV, d=D, k_pool=db.k_pool, v_pool=db.v_pool, q=d_q, out=d_out,
                            requests=db.requests, mode=libape.APE_DECODE)
     ws_d = plan_d.alloc_workspace()
+    # the same decode batch with all 16 requests attending to request 0's contexts: the contexts are read once
+    sb = wl.share_contexts(db)
+    s_out = torch.zeros_like(d_q)
+    plan_s = h.attend_plan(H_q=H_Q, H_kv=H_KV, d=D, k_pool=db.k_pool, v_pool=db.v_pool, q=d_q, out=s_out,
+                           requests=sb.requests, mode=libape.APE_DECODE, shared=True)
+    ws_s = plan_s.alloc_workspace()
 
     fl_prefill = attend_flops(L_Q, L_P, N_CTX * L_CTX, L_Q)
     fl_encode = encode_flops(L_P, [L_CTX] * N_CTX)
@@ -243,6 +250,8 @@ def main():
         if ev: ev[2].record()
         plan_d.attend(db.T, db.S, ws_d)
         if ev: ev[3].record()
+        plan_s.attend(db.T, db.S, ws_s)
+        if ev: ev[5].record()
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -250,7 +259,7 @@ def main():
     assert h.get_status() == 0, "a kernel reported a timed-out wait"
 
     sampler = ClockSampler(local_rank)
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
     if dist:
         td.barrier()
     torch.cuda.synchronize()
@@ -269,8 +278,9 @@ def main():
     t_pre = sum(e[1].elapsed_time(e[2]) for e in events) / args.steps
     t_dec = sum(e[2].elapsed_time(e[3]) for e in events) / args.steps
     t_rope = sum(e[4].elapsed_time(e[0]) for e in events) / args.steps
-    t_step = events[0][4].elapsed_time(events[-1][3]) / args.steps
-    t_enc, t_pre, t_dec, t_step, t_rope = dist_util.max_over_ranks([t_enc, t_pre, t_dec, t_step, t_rope], dev)
+    t_shared = sum(e[3].elapsed_time(e[5]) for e in events) / args.steps
+    t_step = events[0][4].elapsed_time(events[-1][5]) / args.steps
+    t_enc, t_pre, t_dec, t_step, t_rope, t_shared = dist_util.max_over_ranks([t_enc, t_pre, t_dec, t_step, t_rope, t_shared], dev)
 
     # ---- end to end through the host-buffer entry point (prefill half of the metric) ---------------------------------
     e2e = None
@@ -319,10 +329,14 @@ def main():
         "prefill": {"ms": t_pre, "tflops": tf_prefill, "flops": fl_prefill},
         "decode": {"ms_per_step": t_dec, "value": world * gbs_decode, "unit": "GB/s", "bytes": by_decode, "tflops": fl_decode / (t_dec * 1e-3) / 1e12,
                    "roofline": roof_dec},
+        "decode_shared_contexts": {"ms_per_step": t_shared, "speedup_over_decode": t_dec / t_shared,
+                                   "kv_bytes_served": by_decode, "kv_bytes_read": (DEC_REQ * (L_P + DEC_LK) + N_CTX * L_CTX) * 4.0 * H_KV * D,
+                                   "what": "the decode batch with all requests on one set of contexts (ape_attend_plan_shared): contexts read once, "
+                                           "context pass on the tensor cores (64 live rows of a 256-row block)"},
         "rope": {"ms": t_rope, "value": world * gbs_rope, "unit": "GB/s", "bytes": by_rope, "roofline": roof_rope},
         "encode": {"ms": t_enc, "tflops": tf_encode, "flops": fl_encode, "frac_of_sustained_peak": tf_encode / peaks["tf_sustained"]},
         "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
-        "gpu_launches": args.steps * (3 + plan_e.last_launches() + plan_p.last_launches() + plan_d.last_launches()),
+        "gpu_launches": args.steps * (3 + plan_e.last_launches() + plan_p.last_launches() + plan_d.last_launches() + plan_s.last_launches()),
         "wall_s_timed_region": t_wall,
     }
     print(json.dumps(line))

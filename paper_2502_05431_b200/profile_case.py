@@ -21,7 +21,7 @@ from . import libape, workloads as wl
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["prefill", "decode", "encode", "rag", "rope"])
+    ap.add_argument("case", choices=["prefill", "decode", "encode", "rag", "rope", "shared"])
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--n-ctx", type=int, default=250)
     args = ap.parse_args()
@@ -47,6 +47,19 @@ def main():
         ws = plan.alloc_workspace()
         run = lambda: plan.attend(b.T, b.S, ws)
         work = {"bytes": 4 * (64 + args.n_ctx * 256 + 257) * 4.0 * H_kv * d}
+    elif args.case == "shared":
+        # 16 requests decoding over ONE set of n_ctx cached contexts (many-shot prompts shared by a batch of queries)
+        b = wl.share_contexts(wl.config5(n_req=16, steps=4, n_ctx=args.n_ctx, device=dev))
+        q = b.extra["q_steps"][0].contiguous()
+        out = torch.zeros_like(q)
+        plan = h.attend_plan(H_q=H_q, H_kv=H_kv, d=d, k_pool=b.k_pool, v_pool=b.v_pool, q=q, out=out, requests=b.requests,
+                             mode=libape.APE_DECODE, shared=True)
+        ws = plan.alloc_workspace()
+        run = lambda: plan.attend(b.T, b.S, ws)
+        # bytes an unshared decode of the same batch would read (its algorithmic bytes); the shared plan reads the
+        # contexts once
+        work = {"bytes": 16 * (64 + args.n_ctx * 256 + 257) * 4.0 * H_kv * d,
+                "bytes_read_once": (16 * (64 + 257) + args.n_ctx * 256) * 4.0 * H_kv * d}
     elif args.case == "rope":
         # the step in front of the pre-caching attention: n_ctx contexts of 256 tokens behind a 64-token prefix;
         # K rotated (H_kv heads), V copied, Q rotated (H_q heads), all written at their cache rows
