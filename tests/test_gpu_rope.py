@@ -123,3 +123,24 @@ def test_rope_then_encode_matches_the_oracle_pipeline():
     for n, ((s, l), w) in enumerate(zip(rq.ctx, want)):
         if l:
             compare(out[s:s + l].cpu(), w, f"rope+encode ctx {n}")
+
+
+def test_rope_at_the_benchmark_size_sampled_rows():
+    """K (rotated) and V (copied) of 64 + 500 x 256 tokens under position re-use, the shape bench.py times; the oracle
+    checks sampled rows of every kind of run (prefix, first / middle / last context)."""
+    dev = "cuda:0"
+    H, d, theta, n_ctx = 8, 128, 500000.0, 500
+    runs = [(0, 0, 64, 0)] + [(64 + i * 256, 64 + i * 256, 256, 64) for i in range(n_ctx)]
+    n_tok = 64 + n_ctx * 256
+    g = torch.Generator().manual_seed(41)
+    x = torch.randn(n_tok, H, d, generator=g).to(torch.bfloat16)
+    dst = torch.zeros(n_tok, H, d, dtype=torch.bfloat16, device=dev)
+    plan = libape.RopePlan(handle(), d, theta, runs)
+    plan.write(x.to(dev), dst, rotate=True)
+    torch.cuda.synchronize()
+    out = dst.cpu()
+    pos = np.concatenate([np.arange(64)] + [64 + np.arange(256)] * n_ctx)
+    rows = np.unique(np.concatenate([np.arange(0, 80), np.arange(64 + 255, 64 + 258), np.arange(64000, 64300),
+                                     np.arange(n_tok - 300, n_tok)]))
+    _check_rot(out[rows], ro.rope(x[rows], pos[rows], theta), float(x.abs().max()))
+    assert handle().get_status() == 0

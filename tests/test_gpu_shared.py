@@ -60,3 +60,19 @@ def test_shared_plan_rejects_requests_that_do_not_share():
         handle().attend_plan(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=q, out=out, requests=s.requests,
                              mode=libape.APE_DECODE, shared=True)
     assert e.value.code == -1
+
+
+def test_shared_decode_at_the_benchmark_size_sampled_requests():
+    """16 requests over one set of 500 x 256 cached context tokens behind a 64-token prefix, the shape bench.py times;
+    the oracle checks sampled requests at the first and a late decode step."""
+    lens = [[256] * 500] + [[]] * 15                      # only request 0 owns contexts in the pool; the others borrow them
+    b = wl.share_contexts(wl.make_batch(**LLAMA, l_P=64, ctx_lens=lens, l_q=1, l_k=257, capacity=257 + 255, seed=31,
+                                        T=0.9, S=0.9, name="shared_128k"))
+    for t in (0, 255):
+        out, lse, n = gpu_attend(b, libape.APE_DECODE, shared=True, kv_extra=t)
+        assert n == 3
+        for r in (0, 7, 15):
+            rq = b.requests[r]
+            ref = oracle_attend(b, r, l_k=rq.query_kv[1] + t)
+            compare(out[r:r + 1], ref.out.float(), f"shared 128K step {t} req {r}")
+            assert (lse[r:r + 1].double() - ref.lse).abs().max().item() < 2e-3
