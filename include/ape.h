@@ -197,6 +197,30 @@ int ape_decode_noalloc(const ape_shape_t *shape, const ape_kv_pool_t *pool, cons
                        float T, float S, int64_t kv_extra, int device, void *stream, int32_t *device_status);
 
 /*
+ * Context-sharded attend (section "Parallel Encoding": hundreds of contexts, or more context than one GPU holds): each
+ * shard -- another GPU, or another part of one GPU's pool -- holds a subset of the contexts and plans an ordinary attend
+ * over that subset; ape_attend_partial runs the shard and, instead of the merged output, hands out the two segments of
+ * Eq. 5 separately per query row and head: the context segment's own softmax output and the natural-log LSE of its logits
+ * (temperature applied), and the same for the non-context segment (prefix + query, identical on every shard).
+ * The caller gathers o_ctx / lse_ctx of all shards (one all-gather; 4 * (d + 1) bytes per row and head per shard) and
+ * calls ape_merge_shards, which combines the shards' context segments by the hierarchical softmax identity (appendix
+ * "Hierarchical Formula for Softmax Attention"), applies the scaling factor S to the combined context LSE and merges with
+ * the non-context segment (Eq. 5).  The result equals ape_attend over all contexts.  All four arrays are DEVICE, fp32,
+ * caller-owned: o_* [q rows, H_q, d], lse_* [q rows, H_q], indexed like Q; a segment without keys has lse = -inf.
+ * Not available for per-context plans (APE_ERR_MODE).
+ */
+typedef struct { float *o_ctx, *lse_ctx, *o_oth, *lse_oth; } ape_partials_t;
+
+int ape_attend_partial(ape_plan_t plan, float T, int64_t kv_extra, void *workspace, size_t workspace_bytes,
+                       const ape_partials_t *partials, void *stream);
+
+/* o_ctx_all [n_shards, n_rows, H_q, d], lse_ctx_all [n_shards, n_rows, H_q] (shard-major, as an all-gather leaves them);
+ * o_oth / lse_oth of any one shard; out bf16 rows (16-byte aligned like every tensor), lse nullable. */
+int ape_merge_shards(ape_handle_t handle, const ape_shape_t *shape, int64_t n_rows, int32_t n_shards,
+                     const float *o_ctx_all, const float *lse_ctx_all, const float *o_oth, const float *lse_oth,
+                     float S, const ape_rows_t *out, float *lse, void *stream);
+
+/*
  * Rotary position embedding with position re-use, fused with the write into the cache (the step right before
  * ape_encode_contexts: it makes the K, V and Q that the pre-caching attention and, later, ape_attend read).
  *

@@ -738,8 +738,11 @@ int ape_plan_last_launches(ape_plan_t p, int32_t* n) {
     return APE_OK;
 }
 
-int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace, size_t ws_bytes, void* stream_v) {
+static int attend_impl(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace, size_t ws_bytes, void* stream_v,
+                       const ape_partials_t* part) {
     if (!p) return APE_ERR_INVALID_ARG;
+    if (part && (!part->o_ctx || !part->lse_ctx || !part->o_oth || !part->lse_oth)) return APE_ERR_INVALID_ARG;
+    if (part && p->per_context) return APE_ERR_MODE;
     if (p->kind != PLAN_PREFILL && p->kind != PLAN_DECODE && p->kind != PLAN_SHARED) return APE_ERR_MODE;
     if (!(T > 0.f) || !(S > 0.f) || !std::isfinite(T) || !std::isfinite(S)) return APE_ERR_RANGE;
     if (kv_extra < 0 || kv_extra > p->max_kv_extra) return APE_ERR_RANGE;
@@ -781,6 +784,8 @@ int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace
         mp.rows_per_slot = G; mp.tokens_per_block = 1; mp.ws_o = b_o; mp.ws_ml = b_ml;
         mp.ws_o_ctx = a_o; mp.ws_ml_ctx = a_ml; mp.rows_per_slot_ctx = kAttnRows;
         mp.out = rows_desc(p->out); mp.lse_out = p->lse; mp.S = S; mp.G = G; mp.H_q = p->shape.n_q_heads; mp.D = D;
+        mp.part_o_ctx = part ? part->o_ctx : nullptr; mp.part_lse_ctx = part ? part->lse_ctx : nullptr;
+        mp.part_o_oth = part ? part->o_oth : nullptr; mp.part_lse_oth = part ? part->lse_oth : nullptr;
         if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;
         p->last_launches++;
         return APE_OK;
@@ -814,9 +819,38 @@ int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace
     mp.tokens_per_block = rows_per_slot / G; mp.ws_o = ws_o; mp.ws_ml = ws_ml; mp.out = rows_desc(p->out); mp.lse_out = p->lse;
     mp.ws_o_ctx = ws_o; mp.ws_ml_ctx = ws_ml; mp.rows_per_slot_ctx = rows_per_slot;
     mp.S = S; mp.G = G; mp.H_q = p->shape.n_q_heads; mp.D = D;
+    mp.part_o_ctx = part ? part->o_ctx : nullptr; mp.part_lse_ctx = part ? part->lse_ctx : nullptr;
+    mp.part_o_oth = part ? part->o_oth : nullptr; mp.part_lse_oth = part ? part->lse_oth : nullptr;
     if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;
     p->last_launches++;
     return APE_OK;
+}
+
+int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace, size_t ws_bytes, void* stream_v) {
+    return attend_impl(p, T, S, kv_extra, workspace, ws_bytes, stream_v, nullptr);
+}
+
+int ape_attend_partial(ape_plan_t p, float T, int64_t kv_extra, void* workspace, size_t ws_bytes, const ape_partials_t* part,
+                       void* stream_v) {
+    if (!part) return APE_ERR_INVALID_ARG;
+    return attend_impl(p, T, 1.0f, kv_extra, workspace, ws_bytes, stream_v, part);
+}
+
+int ape_merge_shards(ape_handle_t h, const ape_shape_t* shape, int64_t n_rows, int32_t n_shards, const float* o_ctx_all,
+                     const float* lse_ctx_all, const float* o_oth, const float* lse_oth, float S, const ape_rows_t* out,
+                     float* lse, void* stream_v) {
+    if (!h || !o_ctx_all || !lse_ctx_all || !o_oth || !lse_oth || n_rows <= 0 || n_shards <= 0) return APE_ERR_INVALID_ARG;
+    int G = 1; float c = 0.f;
+    int rc = check_shape(shape, &G, &c);              if (rc) return rc;
+    rc = check_rows(out, shape);                      if (rc) return rc;
+    if (out->n_rows < n_rows) return APE_ERR_INVALID_ARG;
+    if (!(S > 0.f) || !std::isfinite(S)) return APE_ERR_RANGE;
+    for (const void* ptr : {static_cast<const void*>(o_ctx_all), static_cast<const void*>(o_oth)}) if (!aligned16(ptr)) return APE_ERR_ALIGN;
+    rc = set_device(h); if (rc) return rc;
+    ShardMergeParams sp;
+    sp.o_ctx = o_ctx_all; sp.lse_ctx = lse_ctx_all; sp.o_oth = o_oth; sp.lse_oth = lse_oth; sp.n_shards = n_shards; sp.n_rows = n_rows;
+    sp.out = rows_desc(*out); sp.lse_out = lse; sp.S = S; sp.H_q = shape->n_q_heads; sp.D = shape->head_dim;
+    return launch_shard_merge(sp, static_cast<cudaStream_t>(stream_v)) == cudaSuccess ? APE_OK : APE_ERR_CUDA;
 }
 
 int ape_encode_contexts(ape_plan_t p, void* workspace, size_t ws_bytes, void* stream_v) {
@@ -1049,6 +1083,7 @@ int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, cons
     mp.groups = reinterpret_cast<const DevMerge*>(base + o_merge); mp.reqs = dp.reqs; mp.items = dp.items; mp.per_context = 0; mp.n_groups = static_cast<int32_t>(m.merge.size());
     mp.rows_per_slot = G; mp.tokens_per_block = 1; mp.ws_o = ws_o; mp.ws_ml = ws_ml; mp.out = rows_desc(*out); mp.lse_out = lse;
     mp.ws_o_ctx = ws_o; mp.ws_ml_ctx = ws_ml; mp.rows_per_slot_ctx = G;
+    mp.part_o_ctx = nullptr; mp.part_lse_ctx = nullptr; mp.part_o_oth = nullptr; mp.part_lse_oth = nullptr;
     mp.S = S; mp.G = G; mp.H_q = shape->n_q_heads; mp.D = D;
     if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;
     if (device_status != nullptr) {

@@ -75,12 +75,36 @@ struct MergeParams {
     int32_t rows_per_slot_ctx;
     RowsDesc out;
     float* lse_out;                  // nullable, [rows, H_q]
+    // When part_o_ctx is set the kernel stops after the per-segment combine and writes each segment's normalised output
+    // (fp32 [rows, H_q, D]) and natural-log LSE (fp32 [rows, H_q]) instead of the merged result: one shard of a
+    // context-sharded attend.
+    float* part_o_ctx;
+    float* part_lse_ctx;
+    float* part_o_oth;
+    float* part_lse_oth;
     float S;
     int32_t G;
     int32_t H_q;
     int32_t D;
 };
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
+
+// Merge of the shards of a context-sharded attend: the context segments of all shards combine by the hierarchical softmax
+// identity, then Eq. 5's scaling factor and the merge with the non-context segment.
+struct ShardMergeParams {
+    const float* o_ctx;              // [n_shards][rows][H_q][D]
+    const float* lse_ctx;            // [n_shards][rows][H_q], natural log
+    const float* o_oth;              // [rows][H_q][D]
+    const float* lse_oth;            // [rows][H_q]
+    int32_t n_shards;
+    int64_t n_rows;
+    RowsDesc out;
+    float* lse_out;                  // nullable
+    float S;
+    int32_t H_q;
+    int32_t D;
+};
+cudaError_t launch_shard_merge(const ShardMergeParams& p, cudaStream_t stream);
 
 // Rotary embedding with position re-use, fused with the copy to its destination.
 constexpr int kRopeChunkTokens = 16;   // tokens per work item

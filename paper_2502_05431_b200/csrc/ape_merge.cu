@@ -117,6 +117,22 @@ __global__ void __launch_bounds__(256) ape_merge_kernel(const MergeParams p)
     }
     combine_segment<VEC>(p.ws_o, p.ws_ml, g.oth_slot0, g.oth_n, g.slot_stride, p.rows_per_slot, row, p.D, lane, Mo, Lo, ao);
 
+    const int h = g.kv_head * p.G + hg;
+    if (p.part_o_ctx != nullptr) {
+        // one shard of a context-sharded attend: hand out the two segments as they are (Eq. 5 form only)
+        const int64_t rh = static_cast<int64_t>(rq.q_row0 + tok) * p.H_q + h;
+        const float ic = (Lc > 0.f) ? 1.f / Lc : 0.f, io = (Lo > 0.f) ? 1.f / Lo : 0.f;
+        #pragma unroll
+        for (int v = 0; v < VEC; ++v) {
+            p.part_o_ctx[rh * p.D + lane * VEC + v] = ac[v] * ic;
+            p.part_o_oth[rh * p.D + lane * VEC + v] = ao[v] * io;
+        }
+        if (lane == 0) {
+            p.part_lse_ctx[rh] = (Lc > 0.f) ? (Mc + fast_log2(Lc)) * kLn2 : -INFINITY;
+            p.part_lse_oth[rh] = (Lo > 0.f) ? (Mo + fast_log2(Lo)) * kLn2 : -INFINITY;
+        }
+        return;
+    }
     const float lse_o = (Lo > 0.f) ? (Mo + fast_log2(Lo)) : -INFINITY;
     const float top = fmaxf(lse_c, lse_o);
     float wc = 0.f, wo = 0.f, lam = -INFINITY;
@@ -127,7 +143,6 @@ __global__ void __launch_bounds__(256) ape_merge_kernel(const MergeParams p)
         wo = (Lo > 0.f) ? eo * inv / Lo : 0.f;
         lam = (top + fast_log2(ec + eo)) * kLn2;
     }
-    const int h = g.kv_head * p.G + hg;
     __nv_bfloat16* dst = p.out.data + static_cast<int64_t>(rq.q_row0 + tok) * p.out.token_stride
                          + static_cast<int64_t>(h) * p.out.head_stride + lane * VEC;
     float r[VEC];
@@ -143,7 +158,68 @@ __global__ void __launch_bounds__(256) ape_merge_kernel(const MergeParams p)
         p.lse_out[static_cast<int64_t>(rq.q_row0 + tok) * p.H_q + h] = lam;
 }
 
+// Shards of a context-sharded attend (each holds a subset of the contexts): LSE_C = log sum_s e^{LSE_s},
+// O_C = sum_s e^{LSE_s - LSE_C} O_s (appendix "Hierarchical Formula for Softmax Attention"), then Eq. 5 as above.
+template <int VEC>
+__global__ void __launch_bounds__(256) ape_shard_merge_kernel(const ShardMergeParams p)
+{
+    constexpr float kLog2e = 1.4426950408889634f;
+    const int64_t warp_global = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp_global >= p.n_rows * p.H_q) return;
+    const int64_t row = warp_global / p.H_q;
+    const int h = static_cast<int>(warp_global - row * p.H_q);
+    float M = -INFINITY, Z = 0.f, acc[VEC];
+    #pragma unroll
+    for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
+    for (int s = 0; s < p.n_shards; ++s) {
+        const int64_t rh = (static_cast<int64_t>(s) * p.n_rows + row) * p.H_q + h;
+        const float l = p.lse_ctx[rh] * kLog2e;
+        if (!(l > -INFINITY)) continue;
+        const float Mn = fmaxf(M, l);
+        const float f_old = fast_exp2(M - Mn), f_new = fast_exp2(l - Mn);
+        #pragma unroll
+        for (int v = 0; v < VEC; ++v) acc[v] = acc[v] * f_old + p.o_ctx[rh * p.D + lane * VEC + v] * f_new;
+        Z = Z * f_old + f_new;
+        M = Mn;
+    }
+    const float lse_c = (Z > 0.f) ? p.S * (M + fast_log2(Z)) : -INFINITY;
+    const int64_t rh = row * p.H_q + h;
+    const float lo_nat = p.lse_oth[rh];
+    const float lse_o = (lo_nat > -INFINITY) ? lo_nat * kLog2e : -INFINITY;
+    const float top = fmaxf(lse_c, lse_o);
+    float wc = 0.f, wo = 0.f, lam = -INFINITY;
+    if (top > -INFINITY) {
+        const float ec = fast_exp2(lse_c - top), eo = fast_exp2(lse_o - top);
+        const float inv = 1.f / (ec + eo);
+        wc = (Z > 0.f) ? ec * inv / Z : 0.f;
+        wo = (lse_o > -INFINITY) ? eo * inv : 0.f;
+        lam = (top + fast_log2(ec + eo)) * kLn2;
+    }
+    __nv_bfloat16* dst = p.out.data + row * p.out.token_stride + static_cast<int64_t>(h) * p.out.head_stride + lane * VEC;
+    float r[VEC];
+    #pragma unroll
+    for (int v = 0; v < VEC; ++v) r[v] = wc * acc[v] + wo * p.o_oth[rh * p.D + lane * VEC + v];
+    if constexpr (VEC == 4) {
+        uint2 pk; pk.x = pack_bf16x2(r[0], r[1]); pk.y = pack_bf16x2(r[2], r[3]);
+        *reinterpret_cast<uint2*>(dst) = pk;
+    } else {
+        *reinterpret_cast<uint32_t*>(dst) = pack_bf16x2(r[0], r[1]);
+    }
+    if (p.lse_out != nullptr && lane == 0) p.lse_out[rh] = lam;
+}
+
 }  // namespace
+
+cudaError_t launch_shard_merge(const ShardMergeParams& p, cudaStream_t stream)
+{
+    const long long warps = static_cast<long long>(p.n_rows) * p.H_q;
+    if (warps == 0) return cudaSuccess;
+    const int blocks = static_cast<int>((warps * 32 + 255) / 256);
+    if (p.D == 128) ape_shard_merge_kernel<4><<<blocks, 256, 0, stream>>>(p);
+    else ape_shard_merge_kernel<2><<<blocks, 256, 0, stream>>>(p);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream)
 {

@@ -20,7 +20,8 @@ APE_PREFILL, APE_DECODE = 0, 1
 EXPORTS = ["ape_create", "ape_destroy", "ape_attend_plan", "ape_encode_plan", "ape_plan_workspace_bytes",
            "ape_plan_destroy", "ape_attend", "ape_encode_contexts", "ape_attend_host", "ape_plan_last_launches",
            "ape_get_status", "ape_status_string", "ape_decode_noalloc", "ape_attend_plan_per_context",
-           "ape_rope_runs_for_request", "ape_rope_plan", "ape_rope_write", "ape_attend_plan_shared"]
+           "ape_rope_runs_for_request", "ape_rope_plan", "ape_rope_write", "ape_attend_plan_shared",
+           "ape_attend_partial", "ape_merge_shards"]
 
 
 class ApeError(RuntimeError):
@@ -48,6 +49,10 @@ class ape_rows_t(C.Structure):
 class ape_request_t(C.Structure):
     _fields_ = [("q_start", C.c_int64), ("q_len", C.c_int64), ("prefix", ape_span_t), ("ctx", C.POINTER(ape_span_t)),
                 ("n_ctx", C.c_int32), ("query_kv", ape_span_t), ("query_kv_capacity", C.c_int64)]
+
+
+class ape_partials_t(C.Structure):
+    _fields_ = [("o_ctx", C.c_void_p), ("lse_ctx", C.c_void_p), ("o_oth", C.c_void_p), ("lse_oth", C.c_void_p)]
 
 
 class ape_rope_run_t(C.Structure):
@@ -90,6 +95,9 @@ def load() -> C.CDLL:
                                                   C.POINTER(C.c_int32)]
         lib.ape_rope_plan.argtypes = [vp, C.c_int32, C.c_double, C.POINTER(ape_rope_run_t), C.c_int32, C.POINTER(vp)]
         lib.ape_rope_write.argtypes = [vp, C.POINTER(ape_rows_t), C.POINTER(ape_rows_t), C.c_int32, C.c_int32, vp]
+        lib.ape_attend_partial.argtypes = [vp, C.c_float, C.c_int64, vp, C.c_size_t, C.POINTER(ape_partials_t), vp]
+        lib.ape_merge_shards.argtypes = [vp, C.POINTER(ape_shape_t), C.c_int64, C.c_int32, vp, vp, vp, vp, C.c_float,
+                                         C.POINTER(ape_rows_t), vp, vp]
         lib.ape_status_string.argtypes = [C.c_int]
         lib.ape_status_string.restype = C.c_char_p
         for name in EXPORTS:
@@ -221,6 +229,18 @@ class Handle:
         return Plan(self, p, (q, out, k_pool, v_pool, lse))
 
 
+def merge_shards(handle: "Handle", *, H_q: int, H_kv: int, d: int, o_ctx_all: torch.Tensor, lse_ctx_all: torch.Tensor,
+                 o_oth: torch.Tensor, lse_oth: torch.Tensor, S: float, out: torch.Tensor, lse: Optional[torch.Tensor] = None,
+                 softmax_scale: float = 0.0, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """ape_merge_shards: o_ctx_all fp32 [n_shards, rows, H_q, d], lse_ctx_all fp32 [n_shards, rows, H_q] (contiguous)."""
+    shape = ape_shape_t(H_q, H_kv, d, softmax_scale)
+    orows = _rows(out)
+    _check(load().ape_merge_shards(handle._h, C.byref(shape), int(o_ctx_all.shape[1]), int(o_ctx_all.shape[0]),
+                                   o_ctx_all.data_ptr(), lse_ctx_all.data_ptr(), o_oth.data_ptr(), lse_oth.data_ptr(), float(S),
+                                   C.byref(orows), lse.data_ptr() if lse is not None else None, _stream_ptr(stream)),
+           "ape_merge_shards")
+
+
 def rope_runs_for_request(request, src_start: int = 0):
     """ape_rope_runs_for_request: [(src_start, dst_start, len, pos0), ...] of one request under position re-use."""
     spans = (ape_span_t * max(len(request.ctx), 1))(*[ape_span_t(int(s), int(l)) for s, l in request.ctx])
@@ -277,6 +297,14 @@ class Plan:
                stream: Optional[torch.cuda.Stream] = None) -> None:
         _check(load().ape_attend(self._p, float(T), float(S), int(kv_extra), workspace.data_ptr(), workspace.numel(),
                                  _stream_ptr(stream)), "ape_attend")
+
+    def attend_partial(self, T: float, workspace: torch.Tensor, o_ctx: torch.Tensor, lse_ctx: torch.Tensor,
+                       o_oth: torch.Tensor, lse_oth: torch.Tensor, kv_extra: int = 0,
+                       stream: Optional[torch.cuda.Stream] = None) -> None:
+        """ape_attend_partial: fp32 device tensors o_* [q rows, H_q, d], lse_* [q rows, H_q] receive this shard's segments."""
+        part = ape_partials_t(o_ctx.data_ptr(), lse_ctx.data_ptr(), o_oth.data_ptr(), lse_oth.data_ptr())
+        _check(load().ape_attend_partial(self._p, float(T), int(kv_extra), workspace.data_ptr(), workspace.numel(),
+                                         C.byref(part), _stream_ptr(stream)), "ape_attend_partial")
 
     def encode_contexts(self, workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> None:
         _check(load().ape_encode_contexts(self._p, workspace.data_ptr() if workspace is not None else None,

@@ -47,3 +47,53 @@ def test_max_over_ranks_two_processes():
 def test_single_process_is_identity_and_rate():
     assert dist_util.max_over_ranks([3.0, 4.0]) == [3.0, 4.0]
     assert dist_util.whole_job_rate(10.0, 4, 2.0) == 4 * 10.0 / 2e-3
+
+
+# ---- context-sharded attend: the sharding table and the all-gather layout ------------------------------------------
+
+def test_shard_contexts_is_a_balanced_partition():
+    lens = [256] * 37 + [1000, 3, 0, 512, 512, 77]
+    for world in (1, 2, 3, 8):
+        table = dist_util.shard_contexts(lens, world)
+        assert sorted(i for t in table for i in t) == list(range(len(lens)))          # every context exactly once
+        loads = [sum(lens[i] for i in t) for t in table]
+        assert max(loads) - min(loads) <= max(lens)                                    # longest-first greedy bound
+    assert dist_util.shard_contexts([], 4) == [[], [], [], []]
+
+
+def _gather_worker(rank: int, world: int, port: int, out):
+    import torch.distributed as td
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    td.init_process_group("gloo", rank=rank, world_size=world)
+    rows, H, d = 3, 2, 4
+    o = torch.full((rows, H, d), float(rank + 1))
+    l = torch.full((rows, H), float(10 * (rank + 1)))
+    o_all, l_all = dist_util.gather_context_partials(o, l)
+    table = dist_util.shard_contexts([5, 9, 2, 7, 7], world)
+    out.put((rank, tuple(o_all.shape), o_all[:, 0, 0, 0].tolist(), tuple(l_all.shape), l_all[:, 0, 0].tolist(), table))
+    td.barrier()
+    td.destroy_process_group()
+
+
+def test_gather_context_partials_two_processes():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_gather_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, o_shape, o_vals, l_shape, l_vals, table in got:
+        assert o_shape == (2, 3, 2, 4) and l_shape == (2, 3, 2)
+        assert o_vals == [1.0, 2.0] and l_vals == [10.0, 20.0]                       # shard-major, rank r at index r
+    assert got[0][5] == got[1][5]                                                    # every rank derives the same table
+
+
+def test_gather_without_a_process_group_is_one_shard():
+    o, l = torch.zeros(2, 3, 4), torch.zeros(2, 3)
+    o_all, l_all = dist_util.gather_context_partials(o, l)
+    assert tuple(o_all.shape) == (1, 2, 3, 4) and tuple(l_all.shape) == (1, 2, 3)
