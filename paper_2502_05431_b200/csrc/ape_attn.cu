@@ -249,6 +249,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t tS = tmem_base + (w ? kColS1 : kColS0);
         const uint32_t tO = tmem_base + (w ? kColO1 : kColO0);
         const uint32_t my_s_full = bar_s_full + 8 * w, my_p_full = bar_p_full + 32 * w, my_o_full = bar_o_full + 8 * w;
+        const uint32_t leader = (lane == 0) ? 1u : 0u;
         auto wait_all = [&](uint32_t bar, uint32_t parity) {
             return __all_sync(0xffffffffu, mbar_wait(bar, parity, &abort_flag, p.status)) != 0;
         };
@@ -261,7 +262,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) {
                 const uint64_t o = static_cast<uint64_t>(((ks >> 2) * kSlabBytes + (ks & 3) * 32) >> 4);
-                mma_ss(tS, q_desc0 + o, k_desc0 + o, kIdescQK, ks > 0);
+                mma_ss_elect(leader, tS, q_desc0 + o, k_desc0 + o, kIdescQK, ks > 0);
             }
         };
         // P is zero past the last key that any row of the block may see, so the product stops there (rounded up to 16).
@@ -269,7 +270,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             #pragma unroll
             for (int k2 = 0; k2 < 2; ++k2) {
                 const int ks = key_quarter * 2 + k2;
-                mma_ts(tO, tS + ks * 8, v_desc0 + static_cast<uint64_t>((ks * 2048) >> 4), kIdescPV,
+                mma_ts_elect(leader, tO, tS + ks * 8, v_desc0 + static_cast<uint64_t>((ks * 2048) >> 4), kIdescPV,
                        (accumulate || ks > 0) ? 1u : 0u);
             }
         };
@@ -277,7 +278,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             #pragma unroll
             for (int k2 = 0; k2 < 2; ++k2) {
                 const int ks = key_quarter * 2 + k2;
-                if (ks * 16 < n16) mma_ts(tO, tS + ks * 8, v_desc0 + static_cast<uint64_t>((ks * 2048) >> 4), kIdescPV,
+                if (ks * 16 < n16) mma_ts_elect(leader, tO, tS + ks * 8, v_desc0 + static_cast<uint64_t>((ks * 2048) >> 4), kIdescPV,
                        (accumulate || ks > 0) ? 1u : 0u);
             }
         };
@@ -306,7 +307,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 for (int qq = 0; qq < 4; ++qq) {                  // P arrives in quarters of 32 keys
                     if (!wait_all(my_p_full + 8 * qq, pcnt & 1)) return false;
                     tc_fence_after();
-                    if (lane == 0) issue_pv(v_desc0, o_started, qq);
+                    issue_pv(v_desc0, o_started, qq);
                     __syncwarp();
                 }
             } else {
@@ -314,12 +315,12 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 for (int qq = 0; qq < 4; ++qq) {
                     if (!wait_all(my_p_full + 8 * qq, pcnt & 1)) return false;
                     tc_fence_after();
-                    if (lane == 0) issue_pv_cut(v_desc0, o_started, qq, prev_n16);
+                    issue_pv_cut(v_desc0, o_started, qq, prev_n16);
                     __syncwarp();
                 }
             }
             if (kNV == 1) {                                       // single V stage: free it at once, the next V load is waiting
-                if (lane == 0) mma_commit(bar_v_empty + 8 * prev_vs);
+                mma_commit_elect(leader, bar_v_empty + 8 * prev_vs);
                 __syncwarp();
             } else {
                 prev_v_release = bar_v_empty + 8 * prev_vs;       // committed after the next S = Q K^T has been issued
@@ -340,7 +341,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 // buffers this one is put off until the next S = Q K^T is on its way (with one buffer that product waits
                 // for the refill, so the commit cannot wait for it).
                 if (q_loads > 0) {
-                    if (QBUF == 1) { if (lane == 0) mma_commit(bar_q_empty); }
+                    if (QBUF == 1) mma_commit_elect(leader, bar_q_empty);
                     else pending_q_release = bar_q_empty + 8 * ((q_loads - 1) % QBUF);
                 }
                 const uint32_t qb = q_loads % QBUF;
@@ -367,13 +368,11 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     o_started = true;
                 }
                 tc_fence_after();
-                if (lane == 0) {
-                    issue_qk(k_base);
-                    mma_commit(my_s_full);                         // first: the softmax threads wait on this one
-                    mma_commit(bar_k_empty + 8 * ksn);
-                    if (prev_v_release) mma_commit(prev_v_release);
-                    if (pending_q_release) mma_commit(pending_q_release);
-                }
+                issue_qk(k_base);
+                mma_commit_elect(leader, my_s_full);               // first: the softmax threads wait on this one
+                mma_commit_elect(leader, bar_k_empty + 8 * ksn);
+                if (prev_v_release) mma_commit_elect(leader, prev_v_release);
+                if (pending_q_release) mma_commit_elect(leader, pending_q_release);
                 prev_v_release = 0; pending_q_release = 0;
                 __syncwarp();
                 {
@@ -388,7 +387,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (!pv_prev(prev_vs, prev_vphase, prev_valid, prev_n16, o_started)) { ok = false; break; }
                 // o_full only: the stage release waits for the next item's first product (nobody needs it sooner than that,
                 // and after the last item nobody needs it at all)
-                if (lane == 0) mma_commit(my_o_full);
+                mma_commit_elect(leader, my_o_full);
                 __syncwarp();
             }
         }
