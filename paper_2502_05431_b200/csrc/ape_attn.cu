@@ -23,7 +23,7 @@ constexpr int kTileN = kAttnTileN;            // 128 keys per tile
 constexpr int kHalfRows = 128;
 constexpr int kThreads = 384;               // three warpgroups; warps 10 and 11 only take part in the register hand-over
 constexpr int kRegsSoftmax = 216;            // registers per thread after the hand-over (two softmax warpgroups)
-constexpr int kRegsOther = 56;               // producer / MMA warpgroup
+constexpr int kRegsOther = 72;               // producer / MMA warpgroup
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr int kNK = 2;                        // K stages
