@@ -308,7 +308,6 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (!wait_all(my_p_full + 8 * qq, pcnt & 1)) return false;
                     tc_fence_after();
                     issue_pv(v_desc0, o_started, qq);
-                    __syncwarp();
                 }
             } else {
                 #pragma unroll
@@ -316,12 +315,10 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (!wait_all(my_p_full + 8 * qq, pcnt & 1)) return false;
                     tc_fence_after();
                     issue_pv_cut(v_desc0, o_started, qq, prev_n16);
-                    __syncwarp();
                 }
             }
             if (kNV == 1) {                                       // single V stage: free it at once, the next V load is waiting
                 mma_commit_elect(leader, bar_v_empty + 8 * prev_vs);
-                __syncwarp();
             } else {
                 prev_v_release = bar_v_empty + 8 * prev_vs;       // committed after the next S = Q K^T has been issued
             }
@@ -374,7 +371,6 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (prev_v_release) mma_commit_elect(leader, prev_v_release);
                 if (pending_q_release) mma_commit_elect(leader, pending_q_release);
                 prev_v_release = 0; pending_q_release = 0;
-                __syncwarp();
                 {
                     int n_keys = tile.n_valid;                     // keys any row of the block may see
                     if (tile.flags & TILE_CAUSAL) n_keys = min(n_keys, g.last_tok + g.off - tile.key_base + 1);
@@ -388,7 +384,6 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 // o_full only: the stage release waits for the next item's first product (nobody needs it sooner than that,
                 // and after the last item nobody needs it at all)
                 mma_commit_elect(leader, my_o_full);
-                __syncwarp();
             }
         }
         if (!ok) {
