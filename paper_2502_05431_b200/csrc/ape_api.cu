@@ -52,6 +52,8 @@ struct ape_plan_s {
     size_t ws_bytes = 0;
     int64_t max_kv_extra = 0;
     CUtensorMap tm_q{}, tm_k{}, tm_v{}, tm_o{};
+    SplitMaps tm_split{};           // encode plans with split_r > 0
+    int split_r = 0;
     bool o_via_tma = false;         // encode plans: tm_o describes the output rows
     int32_t last_launches = 0;
     bool per_context = false;        // merge form: Eq. 5 (false) or Eq. 11-12 (true)
@@ -590,6 +592,11 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
     p->n_sib = 1;
     const int D = shape->head_dim, H_kv = shape->n_kv_heads, tile = kAttnTileN, TB = kAttnRows / G;
 
+    // A prefix that ends inside a tile shares that tile with the head of each context (when the tail is a multiple of 8 rows,
+    // which the 128-byte swizzle of the copy engine asks for): with a 64-token prefix and 256-token contexts that is 8
+    // tiles per context instead of 10.
+    const int split_r = (prefix->len % tile != 0 && (prefix->len % tile) % 8 == 0 && n_ctx > 0) ? static_cast<int>(prefix->len % tile) : 0;
+    p->split_r = split_r;
     HostMeta m;
     try {
         struct Work { DevItem it; long long cost; };
@@ -599,15 +606,38 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
             m.reqs.push_back(dr);
             if (ctx[i].len == 0) continue;
             const int t0 = static_cast<int>(m.tiles.size());
-            add_span_tiles(m.tiles, prefix->start, prefix->len, tile, 0, 0);
-            const int n_pref = static_cast<int>(m.tiles.size()) - t0;
-            add_span_tiles(m.tiles, ctx[i].start, ctx[i].len, tile, TILE_CAUSAL, 0);
+            int n_pref, head = 0;                     // head: context tokens that share a tile with the prefix tail
+            if (split_r > 0) {
+                // whole prefix tiles, then ONE tile = [prefix tail | first 128 - split_r context tokens], then the rest of
+                // the context in whole tiles: no tile slot is spent on padding between prefix and context
+                add_span_tiles(m.tiles, prefix->start, prefix->len - split_r, tile, 0, 0);
+                head = static_cast<int>(std::min<int64_t>(tile - split_r, ctx[i].len));
+                DevTile mt;
+                mt.tok = static_cast<int32_t>(prefix->start + prefix->len - split_r);
+                mt.n_valid = split_r + head; mt.key_base = -split_r; mt.flags = TILE_CAUSAL | TILE_SPLIT;
+                m.tiles.push_back(mt);
+                n_pref = static_cast<int>(m.tiles.size()) - t0;
+                for (int64_t off = tile - split_r; off < ctx[i].len; off += tile) {
+                    DevTile t;
+                    t.tok = static_cast<int32_t>(ctx[i].start + off);
+                    t.n_valid = static_cast<int32_t>(std::min<int64_t>(tile, ctx[i].len - off));
+                    t.key_base = static_cast<int32_t>(off); t.flags = TILE_CAUSAL;
+                    m.tiles.push_back(t);
+                }
+            } else {
+                add_span_tiles(m.tiles, prefix->start, prefix->len, tile, 0, 0);
+                n_pref = static_cast<int>(m.tiles.size()) - t0;
+                add_span_tiles(m.tiles, ctx[i].start, ctx[i].len, tile, TILE_CAUSAL, 0);
+            }
             const int t1 = static_cast<int>(m.tiles.size());
             const int RB = static_cast<int>((ctx[i].len + TB - 1) / TB);
             for (int hh = 0; hh < H_kv; ++hh)
                 for (int rb = 0; rb < RB; ++rb) {
                     const int64_t last_tok = std::min<int64_t>(ctx[i].len, static_cast<int64_t>(rb + 1) * TB) - 1;
-                    const int vis = n_pref + static_cast<int>(last_tok / tile) + 1;     // tiles this row block can see
+                    // tiles this row block can see: the prefix tiles and every context tile whose first key is not past last_tok
+                    const int vis = (split_r > 0)
+                        ? n_pref + ((last_tok >= tile - split_r) ? static_cast<int>((last_tok - (tile - split_r)) / tile) + 1 : 0)
+                        : n_pref + static_cast<int>(last_tok / tile) + 1;
                     DevItem it{};
                     it.req = i; it.kv_head = hh; it.row_block = rb; it.tile_begin = t0; it.tile_end = std::min(t1, t0 + vis);
                     it.slot = 0; it.seg = SEG_FINAL; it.n_sib = 1;
@@ -631,6 +661,12 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
         rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
         if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
         if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
+        if (!rc && split_r > 0) {
+            rc = make_map(h, &p->tm_split.ka, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, split_r);
+            if (!rc) rc = make_map(h, &p->tm_split.kb, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile - split_r);
+            if (!rc) rc = make_map(h, &p->tm_split.va, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, split_r);
+            if (!rc) rc = make_map(h, &p->tm_split.vb, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile - split_r);
+        }
         // Every item of this plan has a row block of its own, so a finished row block may leave through its Q buffer.
         if (!rc) p->o_via_tma = make_map(h, &p->tm_o, out->data, D, shape->n_q_heads, out->n_rows, out->head_stride, out->token_stride,
                                          G, 128 / G) == APE_OK;
@@ -768,8 +804,8 @@ static int attend_impl(ape_plan_t p, float T, float S, int64_t kv_extra, void* w
             ap.out = rows_desc(p->out); ap.lse_out = nullptr; ap.ws_o = a_o; ap.ws_ml = a_ml;
             ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c / T * kLog2e;
             ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = a->n_sib; ap.n_q_bufs = 1; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
-            ap.o_via_tma = 0;
-            if (launch_attn(D, a->tm_q, a->tm_k, a->tm_v, a->tm_q, ap, a->n_cta, a->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
+            ap.o_via_tma = 0; ap.split_r = 0;
+            if (launch_attn(D, a->tm_q, a->tm_k, a->tm_v, a->tm_q, a->tm_split, ap, a->n_cta, a->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
             p->last_launches++;
         }
         DecodeParams dp;
@@ -809,8 +845,8 @@ static int attend_impl(ape_plan_t p, float T, float S, int64_t kv_extra, void* w
         ap.out = rows_desc(p->out); ap.lse_out = nullptr; ap.ws_o = ws_o; ap.ws_ml = ws_ml;
         ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c / T * kLog2e;
         ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = p->n_sib; ap.n_q_bufs = 1; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
-        ap.o_via_tma = 0;
-        if (launch_attn(D, p->tm_q, p->tm_k, p->tm_v, p->tm_q, ap, p->n_cta, p->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
+        ap.o_via_tma = 0; ap.split_r = 0;
+        if (launch_attn(D, p->tm_q, p->tm_k, p->tm_v, p->tm_q, p->tm_split, ap, p->n_cta, p->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
     }
     p->last_launches++;
 
@@ -866,8 +902,8 @@ int ape_encode_contexts(ape_plan_t p, void* workspace, size_t ws_bytes, void* st
     ap.out = rows_desc(p->out); ap.lse_out = p->lse; ap.ws_o = nullptr; ap.ws_ml = nullptr;
     ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c * kLog2e;
     ap.G = p->G; ap.H_q = p->shape.n_q_heads; ap.n_sib = 1; ap.n_q_bufs = 2; ap.q_rows_are_pool = 1; ap.status = p->h->d_status;
-    ap.o_via_tma = p->o_via_tma ? 1 : 0;
-    if (launch_attn(p->shape.head_dim, p->tm_q, p->tm_k, p->tm_v, p->tm_o, ap, p->n_cta, p->smem_bytes,
+    ap.o_via_tma = p->o_via_tma ? 1 : 0; ap.split_r = p->split_r;
+    if (launch_attn(p->shape.head_dim, p->tm_q, p->tm_k, p->tm_v, p->tm_o, p->tm_split, ap, p->n_cta, p->smem_bytes,
                     static_cast<cudaStream_t>(stream_v)) != cudaSuccess) return APE_ERR_CUDA;
     p->last_launches = 1;
     return APE_OK;

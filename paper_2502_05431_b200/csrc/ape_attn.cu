@@ -80,7 +80,8 @@ __device__ __forceinline__ bool tile_visible(const DevTile& t, const ItemGeom& g
 template <int D, int QBUF>
 __global__ void __launch_bounds__(kThreads, 1)
 ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const AttnParams p)
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                const __grid_constant__ SplitMaps tm_split, const AttnParams p)
 {
     constexpr int kSlabs = D / 64;
     constexpr int kTileBytes = kSlabs * kSlabBytes;            // one K or V tile, also one Q half
@@ -202,6 +203,16 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         const int s = kcnt % kNK; const uint32_t use = kcnt / kNK;
                         if (!mbar_wait(bar_k_empty + 8 * s, (use & 1) ^ 1, &abort_flag, p.status)) { ok = false; break; }
                         mbar_expect_tx(bar_k_full + 8 * s, kTileBytes);
+                        if (tile.flags & TILE_SPLIT) {
+                            // prefix tail in the first split_r rows, the context's first tokens behind it: two boxes that
+                            // together fill the tile (same byte count), so no key slot of the tile is wasted on padding
+                            #pragma unroll
+                            for (int sl = 0; sl < kSlabs; ++sl) {
+                                const uint32_t dst = smem_u32(k_smem + s * kTileBytes + sl * kSlabBytes);
+                                tma_load_3d(dst, &tm_split.ka, bar_k_full + 8 * s, sl * 64, item.kv_head, tile.tok);
+                                tma_load_3d(dst + p.split_r * 128, &tm_split.kb, bar_k_full + 8 * s, sl * 64, item.kv_head, item.q_row0);
+                            }
+                        } else
                         #pragma unroll
                         for (int sl = 0; sl < kSlabs; ++sl)
                             tma_load_3d(smem_u32(k_smem + s * kTileBytes + sl * kSlabBytes), &tm_k, bar_k_full + 8 * s,
@@ -212,6 +223,14 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         const int s = vcnt % kNV; const uint32_t use = vcnt / kNV;
                         if (!mbar_wait(bar_v_empty + 8 * s, (use & 1) ^ 1, &abort_flag, p.status)) { ok = false; break; }
                         mbar_expect_tx(bar_v_full + 8 * s, kTileBytes);
+                        if (tile.flags & TILE_SPLIT) {
+                            #pragma unroll
+                            for (int sl = 0; sl < kSlabs; ++sl) {
+                                const uint32_t dst = smem_u32(v_smem + s * kTileBytes + sl * kSlabBytes);
+                                tma_load_3d(dst, &tm_split.va, bar_v_full + 8 * s, sl * 64, item.kv_head, tile.tok);
+                                tma_load_3d(dst + p.split_r * 128, &tm_split.vb, bar_v_full + 8 * s, sl * 64, item.kv_head, item.q_row0);
+                            }
+                        } else
                         #pragma unroll
                         for (int sl = 0; sl < kSlabs; ++sl)
                             tma_load_3d(smem_u32(v_smem + s * kTileBytes + sl * kSlabBytes), &tm_v, bar_v_full + 8 * s,
@@ -708,12 +727,12 @@ cudaError_t attn_set_smem_attr(int D, int q_bufs, size_t smem_bytes) {
 }
 
 cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const CUtensorMap& tm_o,
-                        const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream)
+                        const SplitMaps& split, const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream)
 {
-    if (D == 128 && p.n_q_bufs == 2) ape_attn_kernel<128, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, p);
-    else if (D == 128) ape_attn_kernel<128, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, p);
-    else if (p.n_q_bufs == 2) ape_attn_kernel<64, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, p);
-    else ape_attn_kernel<64, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, p);
+    if (D == 128 && p.n_q_bufs == 2) ape_attn_kernel<128, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
+    else if (D == 128) ape_attn_kernel<128, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
+    else if (p.n_q_bufs == 2) ape_attn_kernel<64, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
+    else ape_attn_kernel<64, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
     return cudaGetLastError();
 }
 

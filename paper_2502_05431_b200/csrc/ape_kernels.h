@@ -48,6 +48,7 @@ struct AttnParams {
     int32_t n_sib;                   // sibling CTAs per group (row blocks that stream the same tiles together)
     int32_t n_q_bufs;                // 1: long items (prefill); 2: many short items (encode), see the kernel
     int32_t q_rows_are_pool;         // encode: Q / O rows are pool tokens (row = context start + i)
+    int32_t split_r;                 // rows of a TILE_SPLIT tile that come from the prefix (a multiple of 8; 0: no such tiles)
     int32_t o_via_tma;               // two-buffer plans whose items all have their own Q: full halves of O leave through shared
                                      // memory (the item's Q buffer) and a bulk tensor store described by tm_o
     int* status;
@@ -55,8 +56,10 @@ struct AttnParams {
 
 size_t attn_smem_bytes(int D, int q_bufs);
 cudaError_t attn_set_smem_attr(int D, int q_bufs, size_t smem_bytes);
+// K and V boxes of split_r rows (prefix part) and 128 - split_r rows (context part) for TILE_SPLIT tiles
+struct SplitMaps { CUtensorMap ka, kb, va, vb; };
 cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const CUtensorMap& tm_o,
-                        const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream);
+                        const SplitMaps& split, const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream);
 
 // Merge of the partials: hierarchical softmax identity inside each segment, then Eq. 5's scaling factor.
 struct MergeParams {

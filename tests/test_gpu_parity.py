@@ -182,6 +182,9 @@ def _check_encode(b):
     dict(**LLAMA, l_P=200, ctx_lens=[[70, 700]]),                                  # prefix longer than a tile; 11 row blocks
     dict(H_q=8, H_kv=8, d=64, l_P=5, ctx_lens=[[300, 17]]),                        # G = 1, d = 64
     dict(H_q=8, H_kv=1, d=128, l_P=130, ctx_lens=[[33, 64, 65]]),                  # G = 8
+    dict(**LLAMA, l_P=64, ctx_lens=[[10, 64, 65, 300, 1]]),                        # prefix tail shares a tile with contexts shorter / longer than the rest of it
+    dict(**LLAMA, l_P=120, ctx_lens=[[7, 8, 9, 200]], gap=2),                      # 8 rows of the shared tile left for the context
+    dict(H_q=8, H_kv=8, d=64, l_P=136, ctx_lens=[[250]]),                          # one whole prefix tile + a tail of 8
 ])
 def test_encode(kw):
     b = wl.make_batch(l_q=1, seed=6, with_encode_q=True, name="encode", **kw)
