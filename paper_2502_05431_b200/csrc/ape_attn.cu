@@ -4,12 +4,16 @@
 // Every item is a run of 128-key tiles of ONE segment, so a plain online softmax per item is exact; the scaling
 // factor S of Eq. 5 acts on whole-segment log-sum-exps and is applied by the merge kernel afterwards.
 //
-// Roles (warp-specialised, 384 threads; warp 11 loads Q in the double-buffered configuration, else idles):
+// Roles (warp-specialised, 384 threads):
 //   warps 0-3 / 4-7  softmax of half 0 / half 1: one thread per row; S is read from TMEM, P = 2^(s - m) goes back
 //                    to TMEM as bf16 over the S columns, the running sum stays in a register; also the epilogue
-//   warp 8           producer: bulk tensor copies of Q, K and V tiles into 128-byte-swizzled shared memory
+//                    (partials to the workspace, final rows to global memory or, for encode, into the item's Q buffer)
+//   warp 8           producer: bulk tensor copies of K and V tiles (and of Q with one Q buffer) into 128-byte-swizzled
+//                    shared memory
 //   warps 9, 10      MMA issuers of half 0 / half 1: S = Q K^T (both operands in shared memory) and O += P V (P from
 //                    TMEM) with tcgen05.mma, accumulators in TMEM; warp 9 owns the TMEM allocation
+//   warp 11          with two Q buffers (encode): loads Q one row block ahead and hands finished O tiles to the bulk
+//                    tensor store; idle otherwise
 // The two halves run one tile apart, so that the tensor pipe works on one half while the other does its exponentials.
 #include "ape_common.cuh"
 #include "ape_kernels.h"
@@ -21,7 +25,7 @@ namespace {
 
 constexpr int kTileN = kAttnTileN;            // 128 keys per tile
 constexpr int kHalfRows = 128;
-constexpr int kThreads = 384;               // three warpgroups; warps 10 and 11 only take part in the register hand-over
+constexpr int kThreads = 384;               // three warpgroups: two of softmax warps, one of producer / issuers / Q loader
 constexpr int kRegsSoftmax = 216;            // registers per thread after the hand-over (two softmax warpgroups)
 constexpr int kRegsOther = 72;               // producer / MMA warpgroup
 constexpr int kProducerWarp = 8;
@@ -159,7 +163,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const bool o_via_tma = (QBUF == 2) && p.o_via_tma != 0;
 
     // Register hand-over at the head of every role: the softmax threads hold a whole 128-column row of S in registers,
-    // the third warpgroup (producer, MMA issuers, one idle warp) gives its share up.
+    // the third warpgroup (producer, MMA issuers, Q loader) gives its share up.
     // Q of one row block (both halves) into buffer n % QBUF, once the MMAs that read that buffer last are done.
     auto load_q = [&](const DevItem& item, const DevReq& rq, const ItemGeom& g, uint32_t n) {
         const uint32_t qb = n % QBUF, q_use = n / QBUF;
