@@ -263,6 +263,14 @@ int ape_rope_write(ape_plan_t plan, const ape_rows_t *src, const ape_rows_t *dst
 /* Kernels launched by the last ape_attend / ape_encode_contexts call on this plan. */
 int ape_plan_last_launches(ape_plan_t plan, int32_t *n_launches);
 
+/*
+ * Self-test of the error path every kernel of the library shares: launches one warp that waits, with the library's
+ * bounded wait, on a barrier nothing ever completes.  After the bound (about a second) the wait gives up, the kernel
+ * returns normally and ape_get_status reports APE_ERR_TIMEOUT; the context stays usable.  Nothing faults, traps or
+ * hangs.  Asynchronous on `stream`.
+ */
+int ape_selftest_timeout(ape_handle_t handle, void *stream);
+
 /* Synchronises the device and returns the device status word (0, or APE_ERR_TIMEOUT) in *device_status; clears it. */
 int ape_get_status(ape_handle_t handle, int32_t *device_status);
 const char *ape_status_string(int status);

@@ -942,6 +942,25 @@ int ape_get_status(ape_handle_t h, int32_t* device_status) {
     return APE_OK;
 }
 
+namespace {
+// One warp waits, with the library's bounded wait, on a barrier that nothing ever completes: after the bound (about a second)
+// the wait gives up, raises the status word and the kernel returns normally.
+__global__ void ape_wait_probe_kernel(int* status) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) { ape::mbar_init(ape::smem_u32(&bar), 1); abort_flag = 0; ape::mbar_fence_init(); }
+    __syncwarp();
+    ape::mbar_wait(ape::smem_u32(&bar), 0, &abort_flag, status);
+}
+}  // namespace
+
+int ape_selftest_timeout(ape_handle_t h, void* stream_v) {
+    if (!h) return APE_ERR_INVALID_ARG;
+    int rc = set_device(h); if (rc) return rc;
+    ape_wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream_v)>>>(h->d_status);
+    return cudaGetLastError() == cudaSuccess ? APE_OK : APE_ERR_CUDA;
+}
+
 const char* ape_status_string(int s) {
     switch (s) {
         case APE_OK: return "ok";

@@ -21,7 +21,7 @@ EXPORTS = ["ape_create", "ape_destroy", "ape_attend_plan", "ape_encode_plan", "a
            "ape_plan_destroy", "ape_attend", "ape_encode_contexts", "ape_attend_host", "ape_plan_last_launches",
            "ape_get_status", "ape_status_string", "ape_decode_noalloc", "ape_attend_plan_per_context",
            "ape_rope_runs_for_request", "ape_rope_plan", "ape_rope_write", "ape_attend_plan_shared",
-           "ape_attend_partial", "ape_merge_shards"]
+           "ape_attend_partial", "ape_merge_shards", "ape_selftest_timeout"]
 
 
 class ApeError(RuntimeError):
@@ -98,6 +98,7 @@ def load() -> C.CDLL:
         lib.ape_attend_partial.argtypes = [vp, C.c_float, C.c_int64, vp, C.c_size_t, C.POINTER(ape_partials_t), vp]
         lib.ape_merge_shards.argtypes = [vp, C.POINTER(ape_shape_t), C.c_int64, C.c_int32, vp, vp, vp, vp, C.c_float,
                                          C.POINTER(ape_rows_t), vp, vp]
+        lib.ape_selftest_timeout.argtypes = [vp, vp]
         lib.ape_status_string.argtypes = [C.c_int]
         lib.ape_status_string.restype = C.c_char_p
         for name in EXPORTS:
@@ -179,6 +180,10 @@ class Handle:
             self.close()
         except Exception:
             pass
+
+    def selftest_timeout(self, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """ape_selftest_timeout: a bounded wait that runs out; get_status() then returns APE_ERR_TIMEOUT (-8) once."""
+        _check(load().ape_selftest_timeout(self._h, _stream_ptr(stream)), "ape_selftest_timeout")
 
     def get_status(self) -> int:
         v = C.c_int32(0)

@@ -251,3 +251,16 @@ def test_prefill_long_query_many_row_blocks():
         compare(out, ref.out.float(), f"long_q rows {rows}")
         sel = ~torch.isnan(ref.lse)
         assert (lse.double()[sel] - ref.lse[sel]).abs().max().item() < 2e-3
+
+
+# ---- the error path of the bounded waits -------------------------------------------------------------------------------
+
+def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    h = handle()
+    assert h.get_status() == 0
+    h.selftest_timeout()                       # one warp waits (bounded, about a second) on a barrier nothing completes
+    assert h.get_status() == -8                # APE_ERR_TIMEOUT, read once ...
+    assert h.get_status() == 0                 # ... and cleared
+    assert libape.status_string(-8)
+    b = wl.make_batch(**LLAMA, l_P=16, ctx_lens=[[64, 64]], l_q=1, l_k=5, seed=77, T=0.9, S=0.9, name="after_timeout")
+    _check_batch(b, libape.APE_DECODE)         # the same context still computes correctly
