@@ -83,9 +83,20 @@ typedef struct {          /* one request (HOST struct; ctx is a HOST array) */
     int64_t query_kv_capacity;     /* >= query_kv.len: pool tokens reserved from query_kv.start for appends    */
 } ape_request_t;
 
-/* Library instance bound to one device.  Allocates a 4-byte device status word.  `device` is a CUDA ordinal. */
+/* Library instance bound to one device.  Allocates a 4-byte device status word.  `device` is a CUDA ordinal.
+ * Every entry point makes its handle's device current while it runs and puts the caller's current device back before
+ * it returns. */
 int ape_create(ape_handle_t *handle, int device);
 int ape_destroy(ape_handle_t handle);
+
+/*
+ * Plans made after this call use at most n_sm thread blocks (one per SM) instead of the whole GPU, e.g. to leave SMs to
+ * a collective or another stream that runs beside the attention; 0 restores the device's SM count.  The split of the
+ * key/value stream over thread blocks (the split-KV of the appendix "Hierarchical Formula for Softmax Attention")
+ * follows the budget, the result does not depend on it beyond rounding.  1 <= n_sm <= SMs of the device, else
+ * APE_ERR_INVALID_ARG.  Plans that already exist keep their split.
+ */
+int ape_set_sm_budget(ape_handle_t handle, int32_t n_sm);
 
 /*
  * Plan an attend over n_req independent requests that share one pool and one Q / O tensor.
@@ -149,7 +160,9 @@ int ape_plan_destroy(ape_plan_t plan);
 int ape_attend(ape_plan_t plan, float T, float S, int64_t kv_extra,
                void *workspace, size_t workspace_bytes, void *stream);
 
-/* Launch the context pre-encoding attention of an encode plan.  No T, no S (they apply to queries only). */
+/* Launch the context pre-encoding attention of an encode plan.  No T, no S (they apply to queries only).  An encode
+ * plan writes its outputs directly and needs no scratch (ape_plan_workspace_bytes gives 0): `workspace` and
+ * `workspace_bytes` are accepted so that all launches look alike, and are ignored (NULL / 0 are fine). */
 int ape_encode_contexts(ape_plan_t plan, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
@@ -162,6 +175,19 @@ int ape_encode_contexts(ape_plan_t plan, void *workspace, size_t workspace_bytes
 int ape_attend_host(ape_plan_t plan, float T, float S, int64_t kv_extra, void *workspace, size_t workspace_bytes,
                     const void *h_q, const void *h_k_pool, const void *h_v_pool, void *h_out,
                     size_t *h2d_bytes, size_t *d2h_bytes, void *stream);
+
+/*
+ * One decode step for callers whose per-step tensors live in HOST memory (the cache itself stays on the device, that is
+ * what makes it a cache).  For a decode plan or a shared-context plan: copies the new token's query rows h_q
+ * [n_req, H_q, d] to the requests' rows of Q; if h_k_new / h_v_new are given (both or neither; [n_req, H_kv, d], dense),
+ * appends them to the requests' query segments at the position step `kv_extra` adds (the "append" that precedes a
+ * decode step: the row of the newest token at planning time + kv_extra); launches ape_attend; copies the requests' rows
+ * of O to h_out [n_req, H_q, d]; synchronises `stream`.  Request r's rows are the r-th of every host array.  Host buffers
+ * should be pinned.  No allocation.  *h2d_bytes / *d2h_bytes (nullable) receive the bytes moved.
+ */
+int ape_decode_step_host(ape_plan_t plan, float T, float S, int64_t kv_extra, void *workspace, size_t workspace_bytes,
+                         const void *h_q, const void *h_k_new, const void *h_v_new, void *h_out,
+                         size_t *h2d_bytes, size_t *d2h_bytes, void *stream);
 
 /*
  * Allocation-free decode step.  (The paper has no counterpart to this entry point; it exists for the callers
@@ -181,16 +207,24 @@ int ape_attend_host(ape_plan_t plan, float T, float S, int64_t kv_extra, void *w
  *     (SMs + 2 * n_req * H_kv) * (H_q / H_kv) * d * 4 bytes of partials).  A larger batch is rejected with
  *     APE_ERR_WORKSPACE before anything is launched; nothing is ever allocated instead.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) and the device's
- *     properties; make that first call outside any stream capture.  With lazy module loading this lookup is also
- *     the moment the runtime materialises the array, so the driver's free-memory figure drops by 8 MiB once.  Later calls only do host work, two
- *     stream-ordered copies/memsets into the array and two kernel launches on `stream`.
+ *     properties.  With lazy module loading this lookup is also the moment the runtime materialises the array, so the
+ *     driver's free-memory figure drops by 8 MiB once.  Later calls only do host work, one stream-ordered copy into the
+ *     array and two kernel launches on `stream`.
+ *   - `stream` must not be capturing: the metadata is rebuilt from the host arrays on every call and uploaded from a
+ *     buffer that dies with the call, so the work cannot be recorded for replay.  A capturing stream is refused with
+ *     APE_ERR_MODE before anything is enqueued.
  *   - Calls no cudaMalloc, cudaFree, or any other allocating routine.  Host descriptors are read during the call.
  *   - All calls on a device share the one array, and it keeps the previous call's contents: each call rewrites
- *     the metadata it uses and clears the status word first.  Two calls whose GPU work may overlap (different
- *     streams, or different threads) race on the array: order them on one stream or with events.
- *   - Asynchronous like ape_attend when `device_status` is NULL.  With a non-NULL `device_status` (HOST pointer)
- *     the call synchronises `stream` after its launches and stores the array's status word there: 0, or
- *     APE_ERR_TIMEOUT if a kernel gave up on a bounded wait.
+ *     the metadata it uses.  Two calls whose GPU work may overlap (different streams, or different threads) race on
+ *     the array: order them on one stream or with events.
+ *   - Host-side blocking: the metadata (16 bytes per 64-token tile, about 0.5 MB for sixteen 128K-token requests) is
+ *     uploaded from pageable host memory, so the call returns only after the work enqueued earlier on `stream` has
+ *     drained and the bytes are staged.  The kernels it launches then run asynchronously, like those of ape_attend.  A
+ *     decode loop that needs the host to run ahead of the GPU plans once with ape_attend_plan instead.
+ *   - Status word: a kernel that gives up on a bounded wait sets the array's status word, and the word STAYS set, also
+ *     across later calls, until a call reads it.  With a non-NULL `device_status` (HOST pointer) the call synchronises
+ *     `stream` after its launches, stores the word there (0 or APE_ERR_TIMEOUT) and clears it.  With NULL nothing is
+ *     read or cleared; a timeout raised by such a call is reported by the next call that passes `device_status`.
  */
 int ape_decode_noalloc(const ape_shape_t *shape, const ape_kv_pool_t *pool, const ape_rows_t *q,
                        const ape_rows_t *out, float *lse, const ape_request_t *requests, int32_t n_req,
@@ -270,9 +304,16 @@ int ape_plan_last_launches(ape_plan_t plan, int32_t *n_launches);
  * hangs.  Asynchronous on `stream`.
  */
 int ape_selftest_timeout(ape_handle_t handle, void *stream);
+/* The same probe aimed at the status word of ape_decode_noalloc's fixed array on `device` (no handle exists there). */
+int ape_selftest_timeout_noalloc(int device, void *stream);
 
-/* Synchronises the device and returns the device status word (0, or APE_ERR_TIMEOUT) in *device_status; clears it. */
+/* Synchronises the WHOLE device (cudaDeviceSynchronize: every stream, also those this library never saw) and returns the
+ * device status word (0, or APE_ERR_TIMEOUT) in *device_status; clears it. */
 int ape_get_status(ape_handle_t handle, int32_t *device_status);
+/* The same for a caller that must not stall its other streams: reads the word in stream order on `stream` and waits for
+ * that stream only, so it reports what the launches enqueued on `stream` before this call have raised.  A word that was
+ * set is cleared by a stream-ordered write on `stream`.  APE_ERR_MODE if `stream` is being captured. */
+int ape_get_status_stream(ape_handle_t handle, void *stream, int32_t *device_status);
 const char *ape_status_string(int status);
 
 #ifdef __cplusplus

@@ -24,7 +24,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 struct ape_handle_s {
     int device = 0;
-    int n_sm = 0;
+    int n_sm = 0;                   // CTAs a plan may use: the device's SM count unless ape_set_sm_budget lowered it
+    int n_sm_device = 0;
     size_t smem_optin = 0;
     int* d_status = nullptr;
     EncodeTiledFn encode_tiled = nullptr;
@@ -60,6 +61,10 @@ struct ape_plan_s {
     // shared-context decode plans: the context pass of all requests (tensor-core kernel) and the per-request rest (decode kernel)
     ape_plan_s* child_ctx = nullptr;
     ape_plan_s* child_oth = nullptr;
+    // decode plans: what the host-buffer step needs (staging for the new token's Q is the plan's Q tensor itself)
+    int n_req = 0;
+    std::vector<int64_t> q_rows;     // Q / O row of every request
+    void* d_step = nullptr;          // [n_req] int64 append rows, then dense staging for the new K and V rows
     // rotary-embedding plans
     RopeChunk* d_rope_chunks = nullptr;
     int n_rope_chunks = 0;
@@ -102,6 +107,9 @@ int check_rows(const ape_rows_t* r, const ape_shape_t* s) {
     if (r->n_rows >= (1ll << 31) - 256) return APE_ERR_LAYOUT;
     return APE_OK;
 }
+
+// the optional fp32 log-sum-exp output: one float per (row, head), so the pointer must be float-aligned
+int check_lse(const float* lse) { return (reinterpret_cast<uintptr_t>(lse) & 3u) ? APE_ERR_ALIGN : APE_OK; }
 
 bool span_ok(const ape_span_t& s, int64_t n_tokens) {
     return s.len >= 0 && s.start >= 0 && s.start <= n_tokens && s.len <= n_tokens - s.start;
@@ -252,7 +260,36 @@ RowsDesc rows_desc(const ape_rows_t& r) {
     RowsDesc d; d.data = static_cast<__nv_bfloat16*>(r.data); d.token_stride = r.token_stride; d.head_stride = r.head_stride; return d;
 }
 
-int set_device(ape_handle_t h) { return cudaSetDevice(h->device) == cudaSuccess ? APE_OK : APE_ERR_CUDA; }
+// Makes `device` current for the lifetime of the object and puts the caller's current device back afterwards: an entry
+// point never leaves a different device current than the one it found.
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int device) {
+        int cur = -1;
+        if (cudaGetDevice(&cur) != cudaSuccess) cur = -1;
+        if (cur == device) { ok = true; return; }
+        ok = cudaSetDevice(device) == cudaSuccess;
+        if (ok) prev = cur;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+    DeviceGuard(const DeviceGuard&) = delete;
+    DeviceGuard& operator=(const DeviceGuard&) = delete;
+};
+
+// Decode plans keep, per request, the pool row of its newest token and a small dense staging area for the K and V rows of
+// the next one, so that a step whose inputs arrive in host memory needs three copies and no allocation.
+int setup_decode_step(ape_plan_t p, const ape_request_t* reqs, int n_req) {
+    p->n_req = n_req;
+    std::vector<int64_t> rows(n_req);
+    p->q_rows.resize(n_req);
+    for (int r = 0; r < n_req; ++r) { rows[r] = reqs[r].query_kv.start + reqs[r].query_kv.len - 1; p->q_rows[r] = reqs[r].q_start; }
+    const size_t b_rows = (static_cast<size_t>(n_req) * 8 + 255) & ~size_t(255);
+    const size_t b_stage = static_cast<size_t>(n_req) * p->shape.n_kv_heads * p->shape.head_dim * 2;
+    if (cudaMalloc(&p->d_step, b_rows + 2 * b_stage) != cudaSuccess) { p->d_step = nullptr; return APE_ERR_NOMEM; }
+    if (cudaMemcpy(p->d_step, rows.data(), static_cast<size_t>(n_req) * 8, cudaMemcpyHostToDevice) != cudaSuccess) return APE_ERR_CUDA;
+    return APE_OK;
+}
 
 }  // namespace
 
@@ -267,10 +304,11 @@ int ape_create(ape_handle_t* handle, int device) {
     ape_handle_t h = new (std::nothrow) ape_handle_s();
     if (!h) return APE_ERR_NOMEM;
     h->device = device;
+    DeviceGuard guard(device);
     cudaDeviceProp prop;
-    if (cudaSetDevice(device) != cudaSuccess || cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete h; return APE_ERR_CUDA; }
+    if (!guard.ok || cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete h; return APE_ERR_CUDA; }
     if (prop.major != 10) { delete h; return APE_ERR_CUDA; }      // the kernels are built for sm_100a only
-    h->n_sm = prop.multiProcessorCount;
+    h->n_sm = h->n_sm_device = prop.multiProcessorCount;
     h->smem_optin = prop.sharedMemPerBlockOptin;
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -284,7 +322,7 @@ int ape_create(ape_handle_t* handle, int device) {
 
 int ape_destroy(ape_handle_t h) {
     if (!h) return APE_ERR_INVALID_ARG;
-    cudaSetDevice(h->device);
+    DeviceGuard guard(h->device);
     if (h->d_status) cudaFree(h->d_status);
     delete h;
     return APE_OK;
@@ -294,7 +332,7 @@ int ape_plan_destroy(ape_plan_t p) {
     if (!p) return APE_ERR_INVALID_ARG;
     if (p->child_ctx) ape_plan_destroy(p->child_ctx);
     if (p->child_oth) ape_plan_destroy(p->child_oth);
-    if (p->d_blob) { cudaSetDevice(p->h->device); cudaFree(p->d_blob); }
+    if (p->d_blob || p->d_step) { DeviceGuard guard(p->h->device); if (p->d_blob) cudaFree(p->d_blob); if (p->d_step) cudaFree(p->d_step); }
     delete p;
     return APE_OK;
 }
@@ -310,6 +348,7 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
     rc = check_pool(pool, shape);                     if (rc) return rc;
     rc = check_rows(q, shape);                        if (rc) return rc;
     rc = check_rows(out, shape);                      if (rc) return rc;
+    rc = check_lse(lse);                              if (rc) return rc;
     if (!reqs || n_req <= 0) return APE_ERR_INVALID_ARG;
     if (mode != APE_PREFILL && mode != APE_DECODE) return APE_ERR_INVALID_ARG;
     if (out->n_rows < q->n_rows) return APE_ERR_INVALID_ARG;
@@ -325,7 +364,8 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
         if (rq.query_kv_capacity < rq.query_kv.len || rq.query_kv.start + rq.query_kv_capacity > pool->n_tokens) return APE_ERR_INVALID_ARG;
         max_extra = std::min(max_extra, rq.query_kv_capacity - rq.query_kv.len);
     }
-    rc = set_device(h); if (rc) return rc;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
 
     ape_plan_t p = new (std::nothrow) ape_plan_s();
     if (!p) return APE_ERR_NOMEM;
@@ -370,12 +410,13 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
             rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
             if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
             if (!rc && decode_set_smem_attr(D, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+            if (!rc) rc = setup_decode_step(p, reqs, n_req);
         } else {
             const int tile = kAttnTileN;
             const int TB = kAttnRows / G;                 // query tokens per row block
             int max_rb = 1;
             for (int r = 0; r < n_req; ++r) max_rb = std::max<int>(max_rb, static_cast<int>((reqs[r].q_len + TB - 1) / TB));
-            p->n_sib = std::min(4, max_rb);
+            p->n_sib = std::max(1, std::min({4, max_rb, h->n_sm}));
             const int n_groups = std::max(1, h->n_sm / p->n_sib);
             for (int r = 0; r < n_req; ++r) {
                 const ape_request_t& rq = reqs[r];
@@ -442,6 +483,7 @@ int ape_attend_plan_shared(ape_handle_t h, const ape_shape_t* shape, const ape_k
     rc = check_pool(pool, shape);                     if (rc) return rc;
     rc = check_rows(q, shape);                        if (rc) return rc;
     rc = check_rows(out, shape);                      if (rc) return rc;
+    rc = check_lse(lse);                              if (rc) return rc;
     if (!reqs || n_req <= 0 || out->n_rows < q->n_rows) return APE_ERR_INVALID_ARG;
     int64_t max_extra = INT64_MAX;
     std::vector<ape_span_t> shared_ctx;
@@ -463,7 +505,8 @@ int ape_attend_plan_shared(ape_handle_t h, const ape_shape_t* shape, const ape_k
                 if (mine[i].start != shared_ctx[i].start || mine[i].len != shared_ctx[i].len) return APE_ERR_INVALID_ARG;
         }
     }
-    rc = set_device(h); if (rc) return rc;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
     const int D = shape->head_dim, H_kv = shape->n_kv_heads;
 
     auto new_plan = [&](PlanKind kind) {
@@ -484,7 +527,7 @@ int ape_attend_plan_shared(ape_handle_t h, const ape_shape_t* shape, const ape_k
         std::vector<Run> runs_a;
         const int TB = kAttnRows / G;
         const int RB = (n_req + TB - 1) / TB;
-        a->n_sib = std::min(4, RB);
+        a->n_sib = std::max(1, std::min({4, RB, h->n_sm}));
         const int n_groups = std::max(1, h->n_sm / a->n_sib);
         ma.reqs.push_back(DevReq{static_cast<int32_t>(reqs[0].q_start), n_req, n_req, 0});
         const int t0 = 0;
@@ -553,6 +596,7 @@ int ape_attend_plan_shared(ape_handle_t h, const ape_shape_t* shape, const ape_k
                     mp.merge.push_back(g);
                 }
             rc = upload(p, mp);
+            if (!rc) rc = setup_decode_step(p, reqs, n_req);
             auto rnd = [](size_t x) { return (x + 255) & ~size_t(255); };
             const size_t rows_a = static_cast<size_t>(a->n_slots) * kAttnRows, rows_b = static_cast<size_t>(b->n_slots) * G;
             a->ws_bytes = rnd(rows_a * D * 4) + rnd(rows_a * 2 * 4);
@@ -578,13 +622,15 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
     rc = check_pool(pool, shape);                     if (rc) return rc;
     rc = check_rows(q, shape);                        if (rc) return rc;
     rc = check_rows(out, shape);                      if (rc) return rc;
+    rc = check_lse(lse);                              if (rc) return rc;
     if (!prefix || n_ctx < 0 || (n_ctx > 0 && !ctx)) return APE_ERR_INVALID_ARG;
     if (!span_ok(*prefix, pool->n_tokens)) return APE_ERR_INVALID_ARG;
     for (int i = 0; i < n_ctx; ++i) {
         if (!span_ok(ctx[i], pool->n_tokens)) return APE_ERR_INVALID_ARG;
         if (ctx[i].start + ctx[i].len > q->n_rows || ctx[i].start + ctx[i].len > out->n_rows) return APE_ERR_INVALID_ARG;
     }
-    rc = set_device(h); if (rc) return rc;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
 
     ape_plan_t p = new (std::nothrow) ape_plan_s();
     if (!p) return APE_ERR_NOMEM;
@@ -704,7 +750,9 @@ int ape_rope_plan(ape_handle_t h, int32_t head_dim, double theta, const ape_rope
     *plan_out = nullptr;
     if (head_dim != 64 && head_dim != 128) return APE_ERR_SHAPE;
     if (!(theta > 1.0) || !std::isfinite(theta)) return APE_ERR_RANGE;
-    int rc = set_device(h); if (rc) return rc;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
+    int rc = APE_OK;
     ape_plan_t p = new (std::nothrow) ape_plan_s();
     if (!p) return APE_ERR_NOMEM;
     p->h = h; p->kind = PLAN_ROPE; p->shape.head_dim = head_dim; p->rope_log2_theta = std::log2(theta);
@@ -748,7 +796,8 @@ int ape_rope_write(ape_plan_t p, const ape_rows_t* src, const ape_rows_t* dst, i
         if (r->head_stride < D || r->token_stride < static_cast<int64_t>(n_heads - 1) * r->head_stride + D) return APE_ERR_INVALID_ARG;
     }
     if (p->rope_src_rows > src->n_rows || p->rope_dst_rows > dst->n_rows) return APE_ERR_INVALID_ARG;
-    int rc = set_device(p->h); if (rc) return rc;
+    DeviceGuard guard(p->h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
     p->last_launches = 0;
     if (p->n_rope_chunks == 0) return APE_OK;
     RopeParams rp;
@@ -783,7 +832,8 @@ static int attend_impl(ape_plan_t p, float T, float S, int64_t kv_extra, void* w
     if (!(T > 0.f) || !(S > 0.f) || !std::isfinite(T) || !std::isfinite(S)) return APE_ERR_RANGE;
     if (kv_extra < 0 || kv_extra > p->max_kv_extra) return APE_ERR_RANGE;
     if (p->ws_bytes > 0 && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || ws_bytes < p->ws_bytes)) return APE_ERR_WORKSPACE;
-    int rc = set_device(p->h); if (rc) return rc;
+    DeviceGuard guard(p->h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const int D = p->shape.head_dim, G = p->G;
     constexpr float kLog2e = 1.4426950408889634f;
@@ -880,9 +930,11 @@ int ape_merge_shards(ape_handle_t h, const ape_shape_t* shape, int64_t n_rows, i
     int rc = check_shape(shape, &G, &c);              if (rc) return rc;
     rc = check_rows(out, shape);                      if (rc) return rc;
     if (out->n_rows < n_rows) return APE_ERR_INVALID_ARG;
+    rc = check_lse(lse);                              if (rc) return rc;
     if (!(S > 0.f) || !std::isfinite(S)) return APE_ERR_RANGE;
     for (const void* ptr : {static_cast<const void*>(o_ctx_all), static_cast<const void*>(o_oth)}) if (!aligned16(ptr)) return APE_ERR_ALIGN;
-    rc = set_device(h); if (rc) return rc;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
     ShardMergeParams sp;
     sp.o_ctx = o_ctx_all; sp.lse_ctx = lse_ctx_all; sp.o_oth = o_oth; sp.lse_oth = lse_oth; sp.n_shards = n_shards; sp.n_rows = n_rows;
     sp.out = rows_desc(*out); sp.lse_out = lse; sp.S = S; sp.H_q = shape->n_q_heads; sp.D = shape->head_dim;
@@ -893,7 +945,8 @@ int ape_encode_contexts(ape_plan_t p, void* workspace, size_t ws_bytes, void* st
     (void)workspace; (void)ws_bytes;
     if (!p) return APE_ERR_INVALID_ARG;
     if (p->kind != PLAN_ENCODE) return APE_ERR_MODE;
-    int rc = set_device(p->h); if (rc) return rc;
+    DeviceGuard guard(p->h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
     p->last_launches = 0;
     if (p->n_items == 0) return APE_OK;
     constexpr float kLog2e = 1.4426950408889634f;
@@ -914,7 +967,9 @@ int ape_attend_host(ape_plan_t p, float T, float S, int64_t kv_extra, void* work
                     size_t* h2d_bytes, size_t* d2h_bytes, void* stream_v) {
     if (!p || !h_q || !h_k || !h_v || !h_out) return APE_ERR_INVALID_ARG;
     if (p->kind != PLAN_PREFILL && p->kind != PLAN_DECODE) return APE_ERR_MODE;
-    int rc = set_device(p->h); if (rc) return rc;
+    DeviceGuard guard(p->h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
+    int rc = APE_OK;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const size_t qb = static_cast<size_t>(p->q.n_rows) * p->q.token_stride * 2;
     const size_t kb = static_cast<size_t>(p->pool.n_tokens) * p->pool.token_stride * 2;
@@ -931,14 +986,95 @@ int ape_attend_host(ape_plan_t p, float T, float S, int64_t kv_extra, void* work
     return APE_OK;
 }
 
+int ape_decode_step_host(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace, size_t ws_bytes,
+                         const void* h_q, const void* h_k_new, const void* h_v_new, void* h_out,
+                         size_t* h2d_bytes, size_t* d2h_bytes, void* stream_v) {
+    if (!p || !h_q || !h_out || (!h_k_new) != (!h_v_new)) return APE_ERR_INVALID_ARG;
+    if ((p->kind != PLAN_DECODE && p->kind != PLAN_SHARED) || !p->d_step) return APE_ERR_MODE;
+    if (kv_extra < 0 || kv_extra > p->max_kv_extra) return APE_ERR_RANGE;
+    DeviceGuard guard(p->h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const int n = p->n_req, H_q = p->shape.n_q_heads, H_kv = p->shape.n_kv_heads, D = p->shape.head_dim;
+    const size_t q_row_bytes = static_cast<size_t>(H_q) * D * 2, kv_row_bytes = static_cast<size_t>(H_kv) * D * 2;
+    // Q rows: one copy when the requests' rows are consecutive and dense, else one strided copy per request
+    bool q_dense = p->q.head_stride == D && p->q.token_stride == static_cast<int64_t>(H_q) * D
+                && p->out.head_stride == D && p->out.token_stride == static_cast<int64_t>(H_q) * D;
+    for (int r = 1; r < n && q_dense; ++r) q_dense = p->q_rows[r] == p->q_rows[0] + r;
+    auto q_ptr = [&](const ape_rows_t& t, int r) { return static_cast<uint8_t*>(t.data) + static_cast<size_t>(p->q_rows[r]) * t.token_stride * 2; };
+    if (q_dense) {
+        if (cudaMemcpyAsync(q_ptr(p->q, 0), h_q, n * q_row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return APE_ERR_CUDA;
+    } else {
+        for (int r = 0; r < n; ++r)
+            if (cudaMemcpy2DAsync(q_ptr(p->q, r), static_cast<size_t>(p->q.head_stride) * 2, static_cast<const uint8_t*>(h_q) + r * q_row_bytes,
+                                  static_cast<size_t>(D) * 2, static_cast<size_t>(D) * 2, H_q, cudaMemcpyHostToDevice, stream) != cudaSuccess) return APE_ERR_CUDA;
+    }
+    size_t up = n * q_row_bytes;
+    if (h_k_new) {
+        // D0: the new token's K and V rows land densely in the plan's staging area and one small kernel puts them at the
+        // rows the query segments have reached (row of the newest token at planning time + kv_extra)
+        uint8_t* base = static_cast<uint8_t*>(p->d_step);
+        const size_t b_rows = (static_cast<size_t>(n) * 8 + 255) & ~size_t(255);
+        uint8_t* k_stage = base + b_rows;
+        uint8_t* v_stage = k_stage + n * kv_row_bytes;
+        if (cudaMemcpyAsync(k_stage, h_k_new, n * kv_row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return APE_ERR_CUDA;
+        if (cudaMemcpyAsync(v_stage, h_v_new, n * kv_row_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return APE_ERR_CUDA;
+        AppendParams ap;
+        ap.k_new = reinterpret_cast<const __nv_bfloat16*>(k_stage); ap.v_new = reinterpret_cast<const __nv_bfloat16*>(v_stage);
+        ap.k_pool = static_cast<__nv_bfloat16*>(const_cast<void*>(p->pool.k)); ap.v_pool = static_cast<__nv_bfloat16*>(const_cast<void*>(p->pool.v));
+        ap.rows = reinterpret_cast<const int64_t*>(base); ap.kv_extra = kv_extra;
+        ap.token_stride = p->pool.token_stride; ap.head_stride = p->pool.head_stride; ap.n_req = n; ap.H_kv = H_kv; ap.D = D;
+        if (launch_append(ap, stream) != cudaSuccess) return APE_ERR_CUDA;
+        up += 2 * n * kv_row_bytes;
+    }
+    int rc = ape_attend(p, T, S, kv_extra, workspace, ws_bytes, stream_v);
+    if (rc) return rc;
+    if (h_k_new) p->last_launches++;
+    if (q_dense) {
+        if (cudaMemcpyAsync(h_out, q_ptr(p->out, 0), n * q_row_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return APE_ERR_CUDA;
+    } else {
+        for (int r = 0; r < n; ++r)
+            if (cudaMemcpy2DAsync(static_cast<uint8_t*>(h_out) + r * q_row_bytes, static_cast<size_t>(D) * 2, q_ptr(p->out, r),
+                                  static_cast<size_t>(p->out.head_stride) * 2, static_cast<size_t>(D) * 2, H_q, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return APE_ERR_CUDA;
+    }
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return APE_ERR_CUDA;
+    if (h2d_bytes) *h2d_bytes = up;
+    if (d2h_bytes) *d2h_bytes = n * q_row_bytes;
+    return APE_OK;
+}
+
 int ape_get_status(ape_handle_t h, int32_t* device_status) {
     if (!h || !device_status) return APE_ERR_INVALID_ARG;
-    int rc = set_device(h); if (rc) return rc;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
     if (cudaDeviceSynchronize() != cudaSuccess) return APE_ERR_CUDA;
     int v = 0;
     if (cudaMemcpy(&v, h->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return APE_ERR_CUDA;
     if (v != 0 && cudaMemset(h->d_status, 0, sizeof(int)) != cudaSuccess) return APE_ERR_CUDA;
     *device_status = v;
+    return APE_OK;
+}
+
+int ape_get_status_stream(ape_handle_t h, void* stream_v, int32_t* device_status) {
+    if (!h || !device_status) return APE_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) return APE_ERR_CUDA;
+    if (cap != cudaStreamCaptureStatusNone) return APE_ERR_MODE;      // a read-back cannot be part of a capture
+    int v = 0;
+    if (cudaMemcpyAsync(&v, h->d_status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return APE_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return APE_ERR_CUDA;
+    // cleared only after it has been copied out, and on the same stream, so a later launch there starts from zero
+    if (v != 0 && cudaMemsetAsync(h->d_status, 0, sizeof(int), stream) != cudaSuccess) return APE_ERR_CUDA;
+    *device_status = v;
+    return APE_OK;
+}
+
+int ape_set_sm_budget(ape_handle_t h, int32_t n_sm) {
+    if (!h || n_sm < 0 || n_sm > h->n_sm_device) return APE_ERR_INVALID_ARG;
+    h->n_sm = (n_sm == 0) ? h->n_sm_device : n_sm;
     return APE_OK;
 }
 
@@ -956,7 +1092,8 @@ __global__ void ape_wait_probe_kernel(int* status) {
 
 int ape_selftest_timeout(ape_handle_t h, void* stream_v) {
     if (!h) return APE_ERR_INVALID_ARG;
-    int rc = set_device(h); if (rc) return rc;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) return APE_ERR_CUDA;
     ape_wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream_v)>>>(h->d_status);
     return cudaGetLastError() == cudaSuccess ? APE_OK : APE_ERR_CUDA;
 }
@@ -1005,7 +1142,8 @@ int noalloc_setup(int device, NoAllocDevice** out) {
     if (device < 0 || device >= kMaxDevices) return APE_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lock(g_noalloc_mutex);
     NoAllocDevice& d = g_noalloc_dev[device];
-    if (cudaSetDevice(device) != cudaSuccess) return APE_ERR_CUDA;
+    DeviceGuard guard(device);
+    if (!guard.ok) return APE_ERR_CUDA;
     if (!d.ready) {
         void* ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return APE_ERR_CUDA;
@@ -1038,29 +1176,44 @@ int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, cons
     rc = check_pool(pool, shape);                     if (rc) return rc;
     rc = check_rows(q, shape);                        if (rc) return rc;
     rc = check_rows(out, shape);                      if (rc) return rc;
+    rc = check_lse(lse);                              if (rc) return rc;
     if (!reqs || n_req <= 0 || out->n_rows < q->n_rows) return APE_ERR_INVALID_ARG;
     if (!(T > 0.f) || !(S > 0.f) || !std::isfinite(T) || !std::isfinite(S)) return APE_ERR_RANGE;
     int64_t max_extra = INT64_MAX, total_tiles = 0;
-    for (int r = 0; r < n_req; ++r) {
-        const ape_request_t& rq = reqs[r];
-        if (rq.q_len != 1 || rq.q_start < 0 || rq.q_start + 1 > q->n_rows) return APE_ERR_INVALID_ARG;
-        if (rq.n_ctx < 0 || (rq.n_ctx > 0 && !rq.ctx)) return APE_ERR_INVALID_ARG;
-        if (!span_ok(rq.prefix, pool->n_tokens) || !span_ok(rq.query_kv, pool->n_tokens)) return APE_ERR_INVALID_ARG;
-        if (rq.query_kv.len < 1) return APE_ERR_INVALID_ARG;
-        if (rq.query_kv_capacity < rq.query_kv.len || rq.query_kv.start + rq.query_kv_capacity > pool->n_tokens) return APE_ERR_INVALID_ARG;
-        total_tiles += (rq.prefix.len + kDecodeTile - 1) / kDecodeTile + (rq.query_kv_capacity + kDecodeTile - 1) / kDecodeTile;
-        for (int i = 0; i < rq.n_ctx; ++i) {
-            if (!span_ok(rq.ctx[i], pool->n_tokens)) return APE_ERR_INVALID_ARG;
-            total_tiles += (rq.ctx[i].len + kDecodeTile - 1) / kDecodeTile;
+    try {
+        for (int r = 0; r < n_req; ++r) {
+            const ape_request_t& rq = reqs[r];
+            if (rq.q_len != 1 || rq.q_start < 0 || rq.q_start + 1 > q->n_rows) return APE_ERR_INVALID_ARG;
+            if (rq.n_ctx < 0 || (rq.n_ctx > 0 && !rq.ctx)) return APE_ERR_INVALID_ARG;
+            if (!span_ok(rq.prefix, pool->n_tokens) || !span_ok(rq.query_kv, pool->n_tokens)) return APE_ERR_INVALID_ARG;
+            if (rq.query_kv.len < 1) return APE_ERR_INVALID_ARG;
+            if (rq.query_kv_capacity < rq.query_kv.len || rq.query_kv.start + rq.query_kv_capacity > pool->n_tokens) return APE_ERR_INVALID_ARG;
+            total_tiles += (rq.prefix.len + kDecodeTile - 1) / kDecodeTile + (rq.query_kv_capacity + kDecodeTile - 1) / kDecodeTile;
+            for (int i = 0; i < rq.n_ctx; ++i) if (!span_ok(rq.ctx[i], pool->n_tokens)) return APE_ERR_INVALID_ARG;
+            // tiles are cut from the fused spans (touching contexts form one span), exactly as the tile list below is
+            for (const auto& sp : fuse_spans(rq.ctx, rq.n_ctx)) total_tiles += (sp.len + kDecodeTile - 1) / kDecodeTile;
+            max_extra = std::min(max_extra, rq.query_kv_capacity - rq.query_kv.len);
         }
-        max_extra = std::min(max_extra, rq.query_kv_capacity - rq.query_kv.len);
+    } catch (const std::bad_alloc&) {
+        return APE_ERR_NOMEM;
     }
     if (kv_extra < 0 || kv_extra > max_extra) return APE_ERR_RANGE;
-    // size gate, before any host vector grows and before anything touches the device
+    // size gate, before the tile list is built and before anything touches the device
     if (static_cast<size_t>(total_tiles) * sizeof(DevTile) > kNoAllocMetaBytes) return APE_ERR_WORKSPACE;
 
     NoAllocDevice* dv = nullptr;
     rc = noalloc_setup(device, &dv);                  if (rc) return rc;
+    DeviceGuard guard(device);
+    if (!guard.ok) return APE_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    {
+        // Never part of a stream capture: the metadata is rebuilt from the caller's host arrays on every call and uploaded
+        // from a buffer that dies with the call, so a replayed graph would read freed host memory and feed the kernels
+        // stale item records.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) return APE_ERR_CUDA;
+        if (cap != cudaStreamCaptureStatusNone) return APE_ERR_MODE;
+    }
     const int D = shape->head_dim, H_kv = shape->n_kv_heads, tile = kDecodeTile;
     const int n_cta = dv->h.n_sm;
 
@@ -1096,7 +1249,7 @@ int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, cons
         const size_t rows = m.items.size() * static_cast<size_t>(G);
         const size_t part_bytes = rnd(rows * D * 4) + rnd(rows * 2 * 4);
         if (meta_end > kNoAllocMetaBytes || part_bytes > kNoAllocBytes - kNoAllocMetaBytes) return APE_ERR_WORKSPACE;
-        blob.assign(meta_end, 0);                                          // byte 0..255: the status word, cleared
+        blob.assign(meta_end, 0);                                          // byte 0..255 stand for the status word: not uploaded
         std::memcpy(blob.data() + o_tiles, m.tiles.data(), m.tiles.size() * sizeof(DevTile));
         std::memcpy(blob.data() + o_items, m.items.data(), m.items.size() * sizeof(DevItem));
         std::memcpy(blob.data() + o_cta, m.cta_begin.data(), m.cta_begin.size() * 4);
@@ -1115,13 +1268,15 @@ int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, cons
     if (!rc) rc = make_map(&dv->h, &tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
     if (rc) return rc;
 
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     unsigned char* base = dv->scratch;
-    // The array still holds the previous call's status word, metadata and partials.  The copy below rewrites the
-    // status word (zero) and all metadata this call uses; partial slots are fully written by the decode kernel before
-    // the merge kernel reads them, so they need no clearing.  The source is pageable host memory: the runtime has
-    // taken its copy of it when cudaMemcpyAsync returns.
-    if (cudaMemcpyAsync(base, blob.data(), blob.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess) return APE_ERR_CUDA;
+    // The array still holds the previous call's status word, metadata and partials.  The copy below rewrites all
+    // metadata this call uses; partial slots are fully written by the decode kernel before the merge kernel reads
+    // them, so they need no clearing.  The status word (first 256 bytes) is NOT rewritten: it is zero when the library
+    // image is loaded, a kernel that gives up on a bounded wait sets it, and it stays set -- across later calls too --
+    // until a call hands it out through `device_status` and clears it.  The source of the copy is pageable host memory:
+    // the runtime waits for earlier work on the stream, stages the bytes, and has taken its copy when the call returns.
+    if (cudaMemcpyAsync(base + o_tiles, blob.data() + o_tiles, blob.size() - o_tiles, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return APE_ERR_CUDA;
 
     constexpr float kLog2e = 1.4426950408889634f;
     const size_t rows = m.items.size() * static_cast<size_t>(G);
@@ -1142,13 +1297,23 @@ int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, cons
     mp.S = S; mp.G = G; mp.H_q = shape->n_q_heads; mp.D = D;
     if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;
     if (device_status != nullptr) {
-        // the caller asked for the status word: this makes the call synchronous
+        // the caller asked for the status word: this makes the call synchronous; a word that was set is cleared once read
         int v = 0;
         if (cudaMemcpyAsync(&v, base, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return APE_ERR_CUDA;
         if (cudaStreamSynchronize(stream) != cudaSuccess) return APE_ERR_CUDA;
+        if (v != 0 && cudaMemsetAsync(base, 0, sizeof(int), stream) != cudaSuccess) return APE_ERR_CUDA;
         *device_status = v;
     }
     return APE_OK;
+}
+
+int ape_selftest_timeout_noalloc(int device, void* stream_v) {
+    NoAllocDevice* dv = nullptr;
+    int rc = noalloc_setup(device, &dv);              if (rc) return rc;
+    DeviceGuard guard(device);
+    if (!guard.ok) return APE_ERR_CUDA;
+    ape_wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream_v)>>>(reinterpret_cast<int*>(dv->scratch));
+    return cudaGetLastError() == cudaSuccess ? APE_OK : APE_ERR_CUDA;
 }
 
 }  // extern "C"

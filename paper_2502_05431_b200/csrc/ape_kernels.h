@@ -127,4 +127,17 @@ struct RopeParams {
 };
 cudaError_t launch_rope(int D, const RopeParams& p, int n_cta, cudaStream_t stream);
 
+// Append of one new token per request to the cache (decode step D0): dense staged rows -> pool rows.
+struct AppendParams {
+    const __nv_bfloat16* k_new;      // [n_req][H_kv][D], dense
+    const __nv_bfloat16* v_new;
+    __nv_bfloat16* k_pool;
+    __nv_bfloat16* v_pool;
+    const int64_t* rows;             // [n_req]: pool row of the newest token when kv_extra = 0
+    int64_t kv_extra;
+    int64_t token_stride, head_stride;
+    int32_t n_req, H_kv, D;
+};
+cudaError_t launch_append(const AppendParams& p, cudaStream_t stream);
+
 }  // namespace ape

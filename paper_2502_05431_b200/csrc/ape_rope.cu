@@ -94,7 +94,29 @@ ape_rope_kernel(const RopeParams p)
     }
 }
 
+// D0 of the decode path: the new token's K and V rows of every request (staged densely, [n_req][H_kv][D]) go to the
+// pool row that the request's query segment has reached.  One thread block per request, 16 bytes per thread and turn.
+__global__ void __launch_bounds__(128) ape_append_kernel(const AppendParams p)
+{
+    const int r = blockIdx.x;
+    const int64_t row = p.rows[r] + p.kv_extra;
+    const int vec_per_head = p.D / 8, n_vec = p.H_kv * vec_per_head;
+    for (int i = threadIdx.x; i < 2 * n_vec; i += blockDim.x) {
+        const int which = i / n_vec, j = i - which * n_vec;
+        const int h = j / vec_per_head, v = j - h * vec_per_head;
+        const __nv_bfloat16* src = (which ? p.v_new : p.k_new) + (static_cast<int64_t>(r) * p.H_kv + h) * p.D + v * 8;
+        __nv_bfloat16* dst = (which ? p.v_pool : p.k_pool) + row * p.token_stride + static_cast<int64_t>(h) * p.head_stride + v * 8;
+        *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_append(const AppendParams& p, cudaStream_t stream) {
+    if (p.n_req <= 0) return cudaSuccess;
+    ape_append_kernel<<<p.n_req, 128, 0, stream>>>(p);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_rope(int D, const RopeParams& p, int n_cta, cudaStream_t stream) {
     if (D == 128) ape_rope_kernel<128><<<n_cta, kRopeThreads, 0, stream>>>(p);

@@ -52,17 +52,24 @@ def gather_context_partials(o_ctx: torch.Tensor, lse_ctx: torch.Tensor):
     w = td.get_world_size()
     o_all = torch.empty((w,) + tuple(o_ctx.shape), dtype=o_ctx.dtype, device=o_ctx.device)
     l_all = torch.empty((w,) + tuple(lse_ctx.shape), dtype=lse_ctx.dtype, device=lse_ctx.device)
-    td.all_gather(list(o_all.unbind(0)), o_ctx.contiguous())      # slab r of the output receives rank r's tensor
-    td.all_gather(list(l_all.unbind(0)), lse_ctx.contiguous())
+    if o_ctx.is_cuda:
+        # NCCL: one collective straight into the shard-major tensor (slab r receives rank r's partials)
+        td.all_gather_into_tensor(o_all, o_ctx.contiguous())
+        td.all_gather_into_tensor(l_all, lse_ctx.contiguous())
+    else:
+        # gloo (CPU ranks) takes the list form; the views are the slabs of the same tensor
+        td.all_gather(list(o_all.unbind(0)), o_ctx.contiguous())
+        td.all_gather(list(l_all.unbind(0)), lse_ctx.contiguous())
     return o_all, l_all
 
 
 def attend_context_sharded(handle, plan, *, H_q: int, H_kv: int, d: int, T: float, S: float, workspace: torch.Tensor,
-                           out: torch.Tensor, lse=None, kv_extra: int = 0) -> None:
+                           out: torch.Tensor, lse=None, kv_extra: int = 0, gather=None) -> None:
     """One context-sharded attend on this rank: `plan` was made over this rank's contexts (see `shard_contexts`), with the
     prefix and the query segment present on every rank.  Runs the local shard (ape_attend_partial), all-gathers the context
     partials (NCCL over NVLink when the tensors are on GPUs; 4 * (d + 1) bytes per row and head per rank) and merges
-    (ape_merge_shards).  Every rank ends up with the full result in `out`."""
+    (ape_merge_shards).  Every rank ends up with the full result in `out`.  `gather` replaces the all-gather (same
+    signature and result layout as `gather_context_partials`), for hosts that bring their own transport."""
     from . import libape
     rows = out.shape[0]
     dev = out.device
@@ -70,6 +77,6 @@ def attend_context_sharded(handle, plan, *, H_q: int, H_kv: int, d: int, T: floa
     l_c = torch.empty((rows, H_q), dtype=torch.float32, device=dev)
     o_o, l_o = torch.empty_like(o_c), torch.empty_like(l_c)
     plan.attend_partial(T, workspace, o_c, l_c, o_o, l_o, kv_extra=kv_extra)
-    o_all, l_all = gather_context_partials(o_c, l_c)
+    o_all, l_all = (gather or gather_context_partials)(o_c, l_c)
     libape.merge_shards(handle, H_q=H_q, H_kv=H_kv, d=d, o_ctx_all=o_all, lse_ctx_all=l_all, o_oth=o_o, lse_oth=l_o, S=S,
                         out=out, lse=lse)

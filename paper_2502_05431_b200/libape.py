@@ -21,7 +21,8 @@ EXPORTS = ["ape_create", "ape_destroy", "ape_attend_plan", "ape_encode_plan", "a
            "ape_plan_destroy", "ape_attend", "ape_encode_contexts", "ape_attend_host", "ape_plan_last_launches",
            "ape_get_status", "ape_status_string", "ape_decode_noalloc", "ape_attend_plan_per_context",
            "ape_rope_runs_for_request", "ape_rope_plan", "ape_rope_write", "ape_attend_plan_shared",
-           "ape_attend_partial", "ape_merge_shards", "ape_selftest_timeout"]
+           "ape_attend_partial", "ape_merge_shards", "ape_selftest_timeout", "ape_selftest_timeout_noalloc",
+           "ape_set_sm_budget", "ape_get_status_stream", "ape_decode_step_host"]
 
 
 class ApeError(RuntimeError):
@@ -86,6 +87,7 @@ def load() -> C.CDLL:
         lib.ape_encode_contexts.argtypes = [vp, vp, C.c_size_t, vp]
         lib.ape_attend_host.argtypes = [vp, C.c_float, C.c_float, C.c_int64, vp, C.c_size_t, vp, vp, vp, vp,
                                         C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), vp]
+        lib.ape_decode_step_host.argtypes = lib.ape_attend_host.argtypes
         lib.ape_plan_last_launches.argtypes = [vp, C.POINTER(C.c_int32)]
         lib.ape_get_status.argtypes = [vp, C.POINTER(C.c_int32)]
         lib.ape_decode_noalloc.argtypes = [C.POINTER(ape_shape_t), C.POINTER(ape_kv_pool_t), C.POINTER(ape_rows_t),
@@ -99,6 +101,9 @@ def load() -> C.CDLL:
         lib.ape_merge_shards.argtypes = [vp, C.POINTER(ape_shape_t), C.c_int64, C.c_int32, vp, vp, vp, vp, C.c_float,
                                          C.POINTER(ape_rows_t), vp, vp]
         lib.ape_selftest_timeout.argtypes = [vp, vp]
+        lib.ape_selftest_timeout_noalloc.argtypes = [C.c_int, vp]
+        lib.ape_set_sm_budget.argtypes = [vp, C.c_int32]
+        lib.ape_get_status_stream.argtypes = [vp, vp, C.POINTER(C.c_int32)]
         lib.ape_status_string.argtypes = [C.c_int]
         lib.ape_status_string.restype = C.c_char_p
         for name in EXPORTS:
@@ -106,6 +111,11 @@ def load() -> C.CDLL:
                 getattr(lib, name).restype = C.c_int
         _lib = lib
     return _lib
+
+
+def selftest_timeout_noalloc(device: int = 0, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """ape_selftest_timeout_noalloc: a bounded wait that runs out and raises the status word of ape_decode_noalloc's array."""
+    _check(load().ape_selftest_timeout_noalloc(int(device), _stream_ptr(stream)), "ape_selftest_timeout_noalloc")
 
 
 def status_string(code: int) -> str:
@@ -189,6 +199,16 @@ class Handle:
         v = C.c_int32(0)
         _check(load().ape_get_status(self._h, C.byref(v)), "ape_get_status")
         return int(v.value)
+
+    def get_status_stream(self, stream: Optional[torch.cuda.Stream] = None) -> int:
+        """ape_get_status_stream: the status word in stream order on `stream`; waits for that stream only."""
+        v = C.c_int32(0)
+        _check(load().ape_get_status_stream(self._h, _stream_ptr(stream), C.byref(v)), "ape_get_status_stream")
+        return int(v.value)
+
+    def set_sm_budget(self, n_sm: int) -> None:
+        """ape_set_sm_budget: later plans use at most n_sm thread blocks (0: the whole device)."""
+        _check(load().ape_set_sm_budget(self._h, int(n_sm)), "ape_set_sm_budget")
 
     def attend_plan(self, *, H_q: int, H_kv: int, d: int, k_pool: torch.Tensor, v_pool: torch.Tensor,
                     q: torch.Tensor, out: torch.Tensor, requests: Sequence, mode: int,
@@ -324,6 +344,18 @@ class Plan:
         _check(load().ape_attend_host(self._p, float(T), float(S), int(kv_extra), workspace.data_ptr(), workspace.numel(),
                                       h_q.data_ptr(), h_k.data_ptr(), h_v.data_ptr(), h_out.data_ptr(),
                                       C.byref(a), C.byref(b), _stream_ptr(stream)), "ape_attend_host")
+        return int(a.value), int(b.value)
+
+    def decode_step_host(self, T: float, S: float, workspace: torch.Tensor, h_q: torch.Tensor, h_out: torch.Tensor,
+                         h_k_new: Optional[torch.Tensor] = None, h_v_new: Optional[torch.Tensor] = None, kv_extra: int = 0,
+                         stream: Optional[torch.cuda.Stream] = None):
+        """ape_decode_step_host: the new token's Q (and optionally its K, V, appended to the cache) from host tensors, O back
+        to a host tensor; returns (h2d_bytes, d2h_bytes)."""
+        a, b = C.c_size_t(0), C.c_size_t(0)
+        _check(load().ape_decode_step_host(self._p, float(T), float(S), int(kv_extra), workspace.data_ptr(), workspace.numel(),
+                                           h_q.data_ptr(), h_k_new.data_ptr() if h_k_new is not None else None,
+                                           h_v_new.data_ptr() if h_v_new is not None else None, h_out.data_ptr(),
+                                           C.byref(a), C.byref(b), _stream_ptr(stream)), "ape_decode_step_host")
         return int(a.value), int(b.value)
 
     def last_launches(self) -> int:

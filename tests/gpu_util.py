@@ -31,13 +31,33 @@ def gpu_attend(b: Batch, mode: int, *, kv_extra: int = 0, want_lse: bool = True,
     lse = torch.full((q.shape[0], b.H_q), float("nan"), dtype=torch.float32, device=dev) if want_lse else None
     plan = handle().attend_plan(H_q=b.H_q, H_kv=b.H_kv, d=b.d, k_pool=k, v_pool=v, q=q, out=out,
                                 requests=b.requests, mode=mode, lse=lse, per_context=per_context, shared=shared)
-    ws = plan.alloc_workspace()
+    ws, check_bands = guarded_workspace(plan)
     plan.attend(b.T, b.S, ws, kv_extra=kv_extra)
     torch.cuda.synchronize()
     assert handle().get_status() == 0
+    check_bands()
     n = plan.last_launches()
     plan.close()
     return out.cpu(), (lse.cpu() if lse is not None else None), n
+
+
+GUARD_BYTES = 4096
+
+
+def guarded_workspace(plan, device=None):
+    """A workspace of exactly the size the plan asks for, with a guard band of GUARD_BYTES on either side that is filled
+    with a byte pattern (0xA5) no kernel writes.  Returns (workspace view, check): check() fails if a launch wrote outside
+    the workspace it was given (the stand-in for a memory checker on the scratch the library owns during a call)."""
+    dev = device if device is not None else torch.device("cuda:0")
+    n = plan.workspace_bytes
+    buf = torch.full((GUARD_BYTES + n + GUARD_BYTES,), 0xA5, dtype=torch.uint8, device=dev)
+    ws = buf[GUARD_BYTES:GUARD_BYTES + max(n, 1)] if n > 0 else buf[GUARD_BYTES:GUARD_BYTES + 256]
+    assert ws.data_ptr() % 256 == 0
+
+    def check():
+        lo, hi = buf[:GUARD_BYTES], buf[GUARD_BYTES + n:] if n > 0 else buf[GUARD_BYTES + 256:]
+        assert bool((lo == 0xA5).all()) and bool((hi == 0xA5).all()), "a kernel wrote outside its workspace"
+    return ws, check
 
 
 def oracle_attend(b: Batch, r: int, *, rows: Optional[Tuple[int, int]] = None, l_k: Optional[int] = None, q_override=None):

@@ -127,26 +127,29 @@ def test_prefill_config3_rag(T, S):
             compare(out[rq.q_start:rq.q_start + rq.q_len], ref.out.float(), f"cfg3 T={T} S={S} req {r} rows {rows}")
 
 
-def test_prefill_config4_manyshot_128k_sampled_rows():
+def test_prefill_config4_manyshot_128k_all_rows():
+    """The 128K many-shot prefill in the launch configuration the benchmark times, every one of its 256 query rows and
+    32 heads against the oracle (output and the log of Eq. 5's denominator)."""
     b = wl.config4()
     out, lse, _ = gpu_attend(b, libape.APE_PREFILL)
     assert not torch.isnan(out.float()).any()
-    for rows in [(0, 2), (127, 129), (254, 256)]:
-        ref = oracle_attend(b, 0, rows=rows)
-        compare(out, ref.out.float(), f"cfg4 rows {rows}")
-        sel = ~torch.isnan(ref.lse)
-        assert (lse.double()[sel] - ref.lse[sel]).abs().max().item() < 2e-3
+    ref = oracle_attend(b, 0)
+    compare(out, ref.out.float(), "cfg4 all rows")
+    for rows in [(0, 64), (64, 128), (128, 192), (192, 256)]:            # no quarter of the row block hides behind the others
+        compare(out[rows[0]:rows[1]], ref.out[rows[0]:rows[1]].float(), f"cfg4 rows {rows}")
+    assert (lse.double() - ref.lse).abs().max().item() < 2e-3
 
 
-def test_decode_config5_128k_sampled_requests():
+def test_decode_config5_128k_all_requests():
+    """Decode at 128K, batch 16, at the first, a middle and the last of the 256 steps: all 16 requests against the oracle."""
     b = wl.config5(n_req=16)
-    dev = torch.device("cuda:0")
     q_steps = b.extra["q_steps"]
     for t in (0, 128, 255):
         out, lse, _ = gpu_attend(b, libape.APE_DECODE, kv_extra=t, q_override=q_steps[t].contiguous())
-        for r in (0, 7, 15):
+        for r in range(16):
             ref = oracle_attend(b, r, l_k=257 + t, q_override=q_steps[t, r:r + 1].contiguous())
             compare(out[r:r + 1], ref.out.float(), f"cfg5 step {t} req {r}")
+            assert (lse[r:r + 1].double() - ref.lse).abs().max().item() < 2e-3
 
 
 # ---- encode -----------------------------------------------------------------------------------------------------------
@@ -191,6 +194,30 @@ def test_encode(kw):
     _check_encode(b)
 
 
+def test_encode_bench_size_500x256():
+    """The encode launch the benchmark times: 500 contexts x 256 tokens behind a 64-token prefix (16,000 work items, more
+    than 100 per CTA, every context through the tile shared with the prefix tail and the bulk-store epilogue).  Every row
+    of every context against the oracle; rows outside the spans must stay untouched."""
+    b = wl.config4(with_encode_q=True)
+    _check_encode(b)
+
+
+def test_encode_many_short_items_per_cta():
+    """600 contexts x 64 tokens behind a 72-token prefix: 4,800 one-row-block items, about 32 per CTA, so every CTA
+    walks both Q buffers many times; the prefix tail (72 rows) shares a tile with 56 of each context's 64 tokens."""
+    b = wl.make_batch(**LLAMA, l_P=72, ctx_lens=[[64] * 600], l_q=1, seed=8, with_encode_q=True, name="encode_many_items")
+    _check_encode(b)
+
+
+def test_encode_many_ragged_items_per_cta():
+    """The same with ragged lengths (row blocks that are not full leave through per-thread stores, full ones through the
+    bulk store, interleaved on the same Q buffers) and a prefix that is no multiple of 8 (no shared tile)."""
+    g = torch.Generator().manual_seed(9)
+    lens = torch.randint(1, 200, (400,), generator=g).tolist()
+    b = wl.make_batch(**LLAMA, l_P=67, ctx_lens=[lens], l_q=1, seed=9, with_encode_q=True, gap=1, name="encode_ragged_items")
+    _check_encode(b)
+
+
 def test_attend_host_matches_attend():
     """The host-buffer entry point (pinned host tensors in and out) gives the same result as the device-pointer one."""
     b = wl.make_batch(**LLAMA, l_P=32, ctx_lens=[[256] * 6], l_q=64, seed=9, T=0.9, S=0.9, name="host")
@@ -206,6 +233,44 @@ def test_attend_host_matches_attend():
     h2d, d2h = plan.attend_host(b.T, b.S, ws, hq, hk, hv, hout)
     assert h2d == hq.numel() * 2 + 2 * hk.numel() * 2 and d2h == hq.numel() * 2
     assert torch.equal(hout, ref)
+    plan.close()
+
+
+def test_decode_step_host_appends_and_attends():
+    """The host-buffer decode step: the new token's Q, K, V come from (pinned) host tensors, K and V are appended to the
+    cache rows the query segment has reached, O comes back to the host.  The device pool starts with NaN in the reserved
+    tail, so a missing or misplaced append cannot go unnoticed.  Three consecutive steps against the oracle."""
+    b = wl.make_batch(**LLAMA, l_P=16, ctx_lens=[[256, 70], [130]], l_q=1, l_k=9, capacity=12, gap=2, seed=14, T=0.9, S=0.8,
+                      name="decode_step_host")
+    dev = torch.device("cuda:0")
+    k, v = b.k_pool.to(dev), b.v_pool.to(dev)
+    for rq in b.requests:                                   # nothing beyond the planned length is on the device yet
+        s0 = rq.query_kv[0] + rq.query_kv[1]
+        k[s0:rq.query_kv[0] + rq.query_kv_capacity] = float("nan")
+        v[s0:rq.query_kv[0] + rq.query_kv_capacity] = float("nan")
+    q = torch.zeros_like(b.q, device=dev)
+    out = torch.full_like(q, float("nan"))
+    plan = handle().attend_plan(H_q=b.H_q, H_kv=b.H_kv, d=b.d, k_pool=k, v_pool=v, q=q, out=out, requests=b.requests,
+                                mode=libape.APE_DECODE)
+    ws = plan.alloc_workspace()
+    g = torch.Generator().manual_seed(15)
+    for t in (0, 1, 2):
+        hq = torch.randn(len(b.requests), b.H_q, b.d, generator=g).to(torch.bfloat16).pin_memory()
+        hout = torch.empty_like(hq).pin_memory()
+        if t == 0:
+            up, down = plan.decode_step_host(b.T, b.S, ws, hq, hout, kv_extra=0)          # the planned tokens are all cached
+            assert up == hq.numel() * 2
+        else:
+            rows = [rq.query_kv[0] + rq.query_kv[1] - 1 + t for rq in b.requests]
+            hk = torch.stack([b.k_pool[r] for r in rows]).contiguous().pin_memory()
+            hv = torch.stack([b.v_pool[r] for r in rows]).contiguous().pin_memory()
+            up, down = plan.decode_step_host(b.T, b.S, ws, hq, hout, h_k_new=hk, h_v_new=hv, kv_extra=t)
+            assert up == hq.numel() * 2 + 2 * hk.numel() * 2
+        assert down == hq.numel() * 2
+        for r, rq in enumerate(b.requests):
+            ref = oracle_attend(b, r, l_k=rq.query_kv[1] + t, q_override=hq[r:r + 1].contiguous())
+            compare(hout[r:r + 1], ref.out.float(), f"decode_step_host step {t} req {r}")
+    assert handle().get_status() == 0
     plan.close()
 
 

@@ -85,3 +85,64 @@ def test_noalloc_decode_asynchronous_form_and_limits():
     with pytest.raises(libape.ApeError) as e:
         libape.decode_noalloc(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=q, out=out, requests=b.requests, T=1.0, S=1.0, kv_extra=5)
     assert e.value.code == -4
+
+
+def test_noalloc_decode_refuses_a_capturing_stream():
+    """The call rebuilds its metadata from host arrays each time, so it can never be recorded into a CUDA graph: on a
+    stream that is being captured it returns APE_ERR_MODE and enqueues nothing."""
+    b = wl.make_batch(**LLAMA, l_P=8, ctx_lens=[[300]], l_q=1, l_k=4, capacity=6, seed=24, T=0.8, S=0.9)
+    dev = torch.device("cuda:0")
+    q, k, v = b.q.to(dev), b.k_pool.to(dev), b.v_pool.to(dev)
+    out = torch.full_like(q, float("nan"))
+    kw = dict(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=q, out=out, requests=b.requests, T=b.T, S=b.S)
+    libape.decode_noalloc(**kw)                       # the one-time set-up happens outside any capture
+    torch.cuda.synchronize()
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        g.capture_begin()
+        try:
+            with pytest.raises(libape.ApeError) as e:
+                libape.decode_noalloc(stream=s, **kw)
+            with pytest.raises(libape.ApeError) as e2:
+                handle().get_status_stream(s)
+        finally:
+            g.capture_end()
+    assert e.value.code == -10 and e2.value.code == -10
+    torch.cuda.synchronize()
+    assert libape.decode_noalloc(want_status=True, **kw) == 0     # and the entry point still works afterwards
+
+
+def test_noalloc_status_word_survives_asynchronous_calls():
+    """A timeout raised on the fixed array stays there until a call reads it: asynchronous calls in between neither report
+    nor erase it."""
+    b = wl.make_batch(**LLAMA, l_P=8, ctx_lens=[[300]], l_q=1, l_k=4, capacity=6, seed=25, T=0.8, S=0.9)
+    dev = torch.device("cuda:0")
+    q, k, v = b.q.to(dev), b.k_pool.to(dev), b.v_pool.to(dev)
+    out = torch.full_like(q, float("nan"))
+    kw = dict(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=q, out=out, requests=b.requests, T=b.T, S=b.S)
+    assert libape.decode_noalloc(want_status=True, **kw) == 0
+    libape.selftest_timeout_noalloc(0)                # one warp whose bounded wait runs out (about a second)
+    assert libape.decode_noalloc(**kw) is None        # asynchronous: does not look at the word
+    assert libape.decode_noalloc(**kw) is None
+    assert libape.decode_noalloc(want_status=True, **kw) == -8
+    assert libape.decode_noalloc(want_status=True, **kw) == 0
+    o_ref, o_new, _, _ = _both(b)
+    _close(o_ref, o_new)
+
+
+def test_noalloc_size_gate_counts_fused_spans():
+    """300,000 one-token contexts that touch each other are ONE span of 300,000 tokens (4,688 tiles): accepted, although
+    300,000 separate tile records would not fit the fixed array."""
+    n = 300000
+    b = wl.make_batch(H_q=4, H_kv=1, d=64, l_P=8, ctx_lens=[[n]], l_q=1, l_k=4, capacity=6, seed=26, T=0.9, S=0.9)
+    rq = b.requests[0]
+    s0 = rq.ctx[0][0]
+    many = wl.Request(rq.q_start, 1, rq.prefix, [(s0 + i, 1) for i in range(n)], rq.query_kv, rq.query_kv_capacity)
+    dev = torch.device("cuda:0")
+    q, k, v = b.q.to(dev), b.k_pool.to(dev), b.v_pool.to(dev)
+    out_a, out_b = torch.full_like(q, float("nan")), torch.full_like(q, float("nan"))
+    kw = dict(H_q=4, H_kv=1, d=64, k_pool=k, v_pool=v, q=q, T=b.T, S=b.S)
+    assert libape.decode_noalloc(out=out_a, requests=[many], want_status=True, **kw) == 0
+    assert libape.decode_noalloc(out=out_b, requests=b.requests, want_status=True, **kw) == 0
+    assert torch.equal(out_a, out_b) and not torch.isnan(out_a.float()).any()
