@@ -11,6 +11,10 @@
  *                        (section "Formulation"), written out per query row, and,
  *                        behind a switch, the per-context hierarchical form of the
  *                        appendix "Hierarchical Formula for APE" (Eq. 11-12).
+ *   ape_oracle_attend_tree : the same attention when the contexts form trees (appendix "Future
+ *                        Directions": each context a tree-like hierarchy, evaluated along each
+ *                        branch with intermediate results merged on the way): the hierarchical
+ *                        formulas of the appendix applied node by node, bottom-up.
  *   ape_oracle_encode  : the block-diagonal attention that pre-caches each
  *                        context (section "Parallel Encoding", pre-caching step,
  *                        with the shared prefix of section "Prepending Shared
@@ -25,6 +29,13 @@
  *     "Efficient Implementation" listing); per_context=1 selects Eq. 11-12.
  *     This choice is pinned by no printed value: PARITY UNPINNED for the choice
  *     between the two readings; each reading itself is pinned by the tests.
+ *   - Context trees: the paper prints no formula for a hierarchy deeper than one level.  Reading
+ *     taken: inside a tree, a node's members (its own tokens and its child nodes) merge by the
+ *     plain hierarchical softmax identity; a node marked as SCALED hands S * LogSumExp to its
+ *     parent, as A^{h'}_{C_i} does in Eq. 11; by default the scaled nodes are the roots, i.e. every
+ *     top-level tree is one context of Eq. 11-12.  PARITY UNPINNED for where S applies along a
+ *     branch; the arithmetic of the reading is pinned by the tests (both ends of the family are
+ *     printed formulas: one tree over everything is Eq. 5, one node per context is Eq. 11-12).
  *   - T applies to context logits only (Eq. 5; the T in the non-context term of
  *     the appendix's "Relation" paragraph is a typo).
  *   - Query rows are causal inside the query segment, bottom-right aligned when
@@ -271,6 +282,130 @@ int ape_oracle_encode(const uint16_t *const *ctx_q, int64_t q_token_stride, int6
                 if (lse && lse[n]) lse[n][(size_t)r * H_q + h] = L;
                 free(qd); free(x);
             }
+        }
+    }
+    return failed ? -2 : 0;
+}
+
+/*
+ * APE attention over context TREES for one request (appendix "Hierarchical Formula for APE" applied along the
+ * branches of the hierarchy sketched in the appendix "Future Directions").
+ *
+ * ctx[n], n = 0..n_ctx-1, are the nodes: node n holds its own tokens (possibly none: a pure grouping node) and has the
+ * parent parent[n], -1 for a top-level node; parent[n] < n, so children always come after their parent.
+ * scaled[n] != 0 marks the nodes that hand S * LogSumExp to their parent (Eq. 11: A^{h'} = S * LogSumExp); the others
+ * hand their LogSumExp unchanged (appendix "Hierarchical Formula for Softmax Attention").
+ *
+ * Per (row, head), level by level:
+ *   1. every node's own tokens: V_own = Softmax(q K_n / (T sqrt(d))) V_n, A_own = LogSumExp(q K_n / (T sqrt(d)));
+ *   2. from the last node to the first (children before parents): the node's members are its own tokens and its
+ *      finished children; A_n = LogSumExp(member A's), V_n = Softmax(member A's) x [member V's]; then the node hands
+ *      (V_n, s_n * A_n) to its parent, s_n = S if scaled[n] else 1;
+ *   3. the final softmax over [A_other, handed A of every top-level node] x [V_other, V of every top-level node],
+ *      A_other / V_other being the non-context segment (prefix + causal query keys), unchanged.
+ * Other arguments and outputs as in ape_oracle_attend; lse is the log of the final softmax's denominator.
+ */
+int ape_oracle_attend_tree(const uint16_t *q, int64_t l_q, int64_t q_token_stride, int64_t q_head_stride,
+                           int H_q, int H_kv, int d, double c,
+                           const orc_kv_t *prefix, const orc_kv_t *ctx, const int32_t *parent, const uint8_t *scaled,
+                           int n_ctx, const orc_kv_t *qkv, double T, double S,
+                           int64_t row_begin, int64_t row_end, int head_begin, int head_end,
+                           double *out, double *lse)
+{
+    if (!q || !out || !prefix || !qkv || H_q <= 0 || H_kv <= 0 || H_q % H_kv || d <= 0) return -1;
+    if (!(T > 0.0) || !(S > 0.0) || n_ctx < 0 || (n_ctx > 0 && (!ctx || !parent || !scaled))) return -1;
+    if (qkv->len < l_q || row_begin < 0 || row_end > l_q || head_begin < 0 || head_end > H_q) return -1;
+    for (int n = 0; n < n_ctx; ++n) if (parent[n] < -1 || parent[n] >= n) return -1;
+
+    const int G = H_q / H_kv;
+    const int64_t l_P = prefix->len, l_k = qkv->len;
+    int64_t max_len = 1;
+    for (int n = 0; n < n_ctx; ++n) if (ctx[n].len > max_len) max_len = ctx[n].len;
+    if (row_end <= row_begin || head_end <= head_begin) return 0;
+    int failed = 0;
+
+    #pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int64_t i = row_begin; i < row_end; ++i) {
+        for (int h = head_begin; h < head_end; ++h) {
+            const int g = h / G;
+            const int64_t n_vis = i + (l_k - l_q) + 1;
+            const int64_t n_oth = l_P + n_vis;
+            double *qd  = (double *)malloc(sizeof(double) * (size_t)d);
+            double *x   = (double *)malloc(sizeof(double) * (size_t)(max_len > n_oth ? max_len : n_oth));
+            double *A   = (double *)malloc(sizeof(double) * (size_t)(n_ctx + 1));        /* [n_ctx]: the non-context segment */
+            double *V   = (double *)malloc(sizeof(double) * (size_t)(n_ctx + 1) * (size_t)d);
+            if (!qd || !x || !A || !V) {
+                #pragma omp atomic write
+                failed = 1;
+                free(qd); free(x); free(A); free(V);
+                continue;
+            }
+            for (int e = 0; e < d; ++e) qd[e] = bf16_to_f64(q[i * q_token_stride + h * q_head_stride + e]);
+
+            /* step 1: every node's own tokens, tempered logits */
+            for (int n = 0; n < n_ctx; ++n) {
+                double *Vn = V + (size_t)n * d;
+                for (int e = 0; e < d; ++e) Vn[e] = 0.0;
+                for (int64_t j = 0; j < ctx[n].len; ++j)
+                    x[j] = (c / T) * dot_qk(qd, ctx[n].k + j * ctx[n].token_stride + g * ctx[n].head_stride, d);
+                A[n] = logsumexp(x, ctx[n].len);
+                for (int64_t j = 0; j < ctx[n].len; ++j) {
+                    const double w = exp(x[j] - A[n]);
+                    const uint16_t *vr = ctx[n].v + j * ctx[n].token_stride + g * ctx[n].head_stride;
+                    for (int e = 0; e < d; ++e) Vn[e] += w * bf16_to_f64(vr[e]);
+                }
+            }
+            /* the non-context segment: prefix keys, then the causal query keys, plain scale */
+            {
+                double *Vo = V + (size_t)n_ctx * d;
+                for (int e = 0; e < d; ++e) Vo[e] = 0.0;
+                for (int64_t j = 0; j < l_P; ++j)
+                    x[j] = c * dot_qk(qd, prefix->k + j * prefix->token_stride + g * prefix->head_stride, d);
+                for (int64_t j = 0; j < n_vis; ++j)
+                    x[l_P + j] = c * dot_qk(qd, qkv->k + j * qkv->token_stride + g * qkv->head_stride, d);
+                A[n_ctx] = logsumexp(x, n_oth);
+                for (int64_t j = 0; j < n_oth; ++j) {
+                    const double w = exp(x[j] - A[n_ctx]);
+                    const uint16_t *vr = (j < l_P) ? prefix->v + j * prefix->token_stride + g * prefix->head_stride
+                                                   : qkv->v + (j - l_P) * qkv->token_stride + g * qkv->head_stride;
+                    for (int e = 0; e < d; ++e) Vo[e] += w * bf16_to_f64(vr[e]);
+                }
+            }
+            /* step 2: bottom-up.  When node n is reached every child of it (index > n) has been finished and has
+             * already been merged into n, one child at a time: merging [own, child_1, ..., child_k] by one softmax
+             * equals merging them pairwise (the identity is associative), and at this point A[n] / V[n] hold node n's
+             * own tokens and all its children.  Finish n and hand it to its parent. */
+            for (int n = n_ctx - 1; n >= 0; --n) {
+                const double handed = (scaled[n] && !(isinf(A[n]) && A[n] < 0)) ? S * A[n] : A[n];
+                A[n] = handed;
+                const int par = parent[n];
+                if (par < 0) continue;
+                const double An = logaddexp(A[par], handed);
+                double *Vp = V + (size_t)par * d, *Vn = V + (size_t)n * d;
+                if (!(isinf(An) && An < 0)) {
+                    const double wp = (isinf(A[par]) && A[par] < 0) ? 0.0 : exp(A[par] - An);
+                    const double wn = (isinf(handed) && handed < 0) ? 0.0 : exp(handed - An);
+                    for (int e = 0; e < d; ++e) Vp[e] = wp * Vp[e] + wn * Vn[e];
+                }
+                A[par] = An;
+            }
+            /* step 3: the final softmax over the non-context segment and the top-level nodes */
+            double Lambda = A[n_ctx];
+            for (int n = 0; n < n_ctx; ++n) if (parent[n] < 0) Lambda = logaddexp(Lambda, A[n]);
+            double *o = out + ((size_t)i * H_q + h) * (size_t)d;
+            {
+                const double w = exp(A[n_ctx] - Lambda);
+                const double *Vo = V + (size_t)n_ctx * d;
+                for (int e = 0; e < d; ++e) o[e] = w * Vo[e];
+            }
+            for (int n = 0; n < n_ctx; ++n) {
+                if (parent[n] >= 0 || (isinf(A[n]) && A[n] < 0)) continue;
+                const double w = exp(A[n] - Lambda);
+                const double *Vn = V + (size_t)n * d;
+                for (int e = 0; e < d; ++e) o[e] += w * Vn[e];
+            }
+            if (lse) lse[(size_t)i * H_q + h] = Lambda;
+            free(qd); free(x); free(A); free(V);
         }
     }
     return failed ? -2 : 0;

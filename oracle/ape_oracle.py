@@ -51,6 +51,11 @@ def _load():
             C.POINTER(C.c_void_p), C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_double,
             C.POINTER(_KV), C.POINTER(_KV), C.c_int, C.c_int64, C.c_int64,
             C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]
+        lib.ape_oracle_attend_tree.restype = C.c_int
+        lib.ape_oracle_attend_tree.argtypes = [
+            C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_double,
+            C.POINTER(_KV), C.POINTER(_KV), C.POINTER(C.c_int32), C.POINTER(C.c_uint8), C.c_int, C.POINTER(_KV),
+            C.c_double, C.c_double, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         lib.ape_oracle_num_threads.restype = C.c_int
         _lib = lib
     return _lib
@@ -119,6 +124,45 @@ def attend(q: torch.Tensor,
     if rc != 0:
         raise RuntimeError(f"ape_oracle_attend failed with code {rc}")
     return AttendResult(out, lse, lse_ctx, wsum)
+
+
+def attend_tree(q: torch.Tensor,
+                prefix: Tuple[torch.Tensor, torch.Tensor],
+                ctx: Sequence[Tuple[torch.Tensor, torch.Tensor]],
+                query_kv: Tuple[torch.Tensor, torch.Tensor],
+                T: float, S: float, parent: Sequence[int], scaled: Optional[Sequence[int]] = None, *,
+                scale: Optional[float] = None, rows: Optional[Tuple[int, int]] = None) -> AttendResult:
+    """APE attention over context trees.  ctx[n] holds node n's own tokens (may be empty), parent[n] < n is its parent
+    (-1: top level); scaled[n] marks the nodes that hand S * LogSumExp upward (default: the top-level nodes).
+    Returns out and lse (lse_ctx and wsum are NaN: not defined for this form)."""
+    lib = _load()
+    _check_bf16_cpu(q, "q")
+    l_q, H_q, d = q.shape
+    H_kv = query_kv[0].shape[1]
+    c = float(scale) if scale is not None else d ** -0.5
+    n = len(ctx)
+    if len(parent) != n:
+        raise ValueError("one parent per node")
+    if scaled is None:
+        scaled = [1 if p < 0 else 0 for p in parent]
+    pk = _kv(prefix[0], prefix[1], "prefix")
+    qk = _kv(query_kv[0], query_kv[1], "query_kv")
+    arr = (_KV * max(n, 1))()
+    for i, (k, v) in enumerate(ctx):
+        arr[i] = _kv(k, v, f"ctx[{i}]")
+    par = (C.c_int32 * max(n, 1))(*[int(p) for p in parent])
+    sc = (C.c_uint8 * max(n, 1))(*[1 if s else 0 for s in scaled])
+    r0, r1 = rows if rows is not None else (0, l_q)
+    out = torch.full((l_q, H_q, d), float("nan"), dtype=torch.float64)
+    lse = torch.full((l_q, H_q), float("nan"), dtype=torch.float64)
+    nan = torch.full((l_q, H_q), float("nan"), dtype=torch.float64)
+    q_ts = q.stride(0) if l_q > 1 else H_q * d
+    q_hs = q.stride(1) if H_q > 1 else d
+    rc = lib.ape_oracle_attend_tree(q.data_ptr(), l_q, q_ts, q_hs, H_q, H_kv, d, c, C.byref(pk), arr, par, sc, n, C.byref(qk),
+                                    float(T), float(S), r0, r1, 0, H_q, out.data_ptr(), lse.data_ptr())
+    if rc != 0:
+        raise RuntimeError(f"ape_oracle_attend_tree failed with code {rc}")
+    return AttendResult(out, lse, nan, nan.clone())
 
 
 def encode(ctx_q: Sequence[torch.Tensor],

@@ -125,6 +125,54 @@ def per_context(q, prefix, ctx, qkv, T, S, scale=None):
     return out
 
 
+def tree_bias(q, prefix, ctx, qkv, T, S, parent, scaled=None, scale=None):
+    """Context trees as ONE dense softmax over the concatenation [P | node_0 .. node_N-1 | Q]: with Z_n the mass of node n
+    (its own tempered weights plus Z_c^{s_c} of every child c) and s_n = S on scaled nodes, 1 elsewhere, a token of node n
+    carries its tempered logit plus (s_m - 1) * log Z_m for every node m on the path from n up to its root: each level's
+    softmax weight Z_m^{s_m} / Z_parent written as a bias.  Returns (out, log of the denominator)."""
+    Q, KP, VP, KC, VC, KQ, VQ = _gather(q, prefix, ctx, qkv)
+    n = len(ctx)
+    if scaled is None:
+        scaled = [1 if p < 0 else 0 for p in parent]
+    s = [S if scaled[i] else 1.0 for i in range(n)]
+    lens = [k.shape[0] for k, _ in ctx]
+    offs = np.concatenate([[0], np.cumsum(lens)]).astype(int)
+    l_q, H_q, d = Q.shape
+    G = H_q // KQ.shape[1]
+    c = d ** -0.5 if scale is None else scale
+    l_P, L_C, l_k = KP.shape[0], KC.shape[0], KQ.shape[0]
+    children = [[j for j in range(n) if parent[j] == i] for i in range(n)]
+    out = np.zeros((l_q, H_q, d))
+    lam = np.zeros((l_q, H_q))
+    mask = _causal_mask(l_q, l_k)
+    for h in range(H_q):
+        g = h // G
+        K = np.concatenate([KP[:, g], KC[:, g], KQ[:, g]], axis=0)
+        V = np.concatenate([VP[:, g], VC[:, g], VQ[:, g]], axis=0)
+        X = c * (Q[:, h] @ K.T)
+        XC = X[:, l_P:l_P + L_C] / T
+        logZ = [None] * n
+
+        def mass(i):                       # log Z_i per row, by its definition (recursion over the children)
+            if logZ[i] is None:
+                terms = [XC[:, offs[i]:offs[i + 1]]] + [(s[j] * mass(j))[:, None] for j in children[i]]
+                logZ[i] = _lse(np.concatenate(terms, axis=1)) if sum(t.shape[1] for t in terms) else np.full(l_q, -np.inf)
+            return logZ[i]
+        bias = np.zeros((l_q, L_C))
+        for i in range(n):
+            m = i
+            while m >= 0:
+                z = mass(m)
+                if lens[i]:
+                    bias[:, offs[i]:offs[i + 1]] += ((s[m] - 1.0) * z)[:, None]
+                m = parent[m]
+        X[:, l_P:l_P + L_C] = XC + bias
+        X[:, l_P + L_C:] = np.where(mask, X[:, l_P + L_C:], -np.inf)
+        out[:, h] = _softmax(X) @ V
+        lam[:, h] = _lse(X)
+    return out, lam
+
+
 def encode_blockdiag(ctx_q, prefix, ctx, scale=None):
     """One dense masked softmax over [P | C_1 | ... | C_N] for all context rows at once."""
     KP, VP = _f64(prefix[0]), _f64(prefix[1])
