@@ -396,6 +396,17 @@ def main():
     plan_pc = h.attend_plan(**kw, k_pool=pb.k_pool, v_pool=pb.v_pool, q=pb.q, out=p_out, requests=pb.requests, mode=libape.APE_PREFILL,
                             per_context=True)
     ws_pc = plan_pc.alloc_workspace()
+    # the same prefill over a two-level context tree: 50 top-level documents (grouping nodes) of 10 chunks each, S per document
+    t_nodes, t_par = [], []
+    for doc in range(N_CTX // 10):
+        t_nodes.append((rq.ctx[0][0], 0)); t_par.append(-1)
+        root = len(t_nodes) - 1
+        for ch in range(10):
+            t_nodes.append(rq.ctx[doc * 10 + ch]); t_par.append(root)
+    t_req = wl.Request(rq.q_start, rq.q_len, rq.prefix, t_nodes, rq.query_kv, rq.query_kv_capacity)
+    plan_t = h.attend_plan(**kw, k_pool=pb.k_pool, v_pool=pb.v_pool, q=pb.q, out=p_out, requests=[t_req], mode=libape.APE_PREFILL,
+                           tree=([t_par], None))
+    ws_t = plan_t.alloc_workspace()
     e_out = torch.zeros_like(pb.q_enc)
     plan_e = h.encode_plan(**kw, k_pool=pb.k_pool, v_pool=pb.v_pool, q=pb.q_enc, out=e_out, prefix=rq.prefix, ctx=rq.ctx)
     # raw (un-rotated) K, V, Q of the prefix and the contexts, packed in request order; the rope leg writes them into the
@@ -434,7 +445,7 @@ def main():
     fl_prefill = attend_flops(L_Q, L_P, N_CTX * L_CTX, L_Q)
     fl_encode = encode_flops(L_P, [L_CTX] * N_CTX)
     dec_tokens = lambda t: L_P + N_CTX * L_CTX + DEC_LK + t
-    legs = ["rope", "encode", "prefill", "decode", "shared", "rag", "per_context"]
+    legs = ["rope", "encode", "prefill", "decode", "shared", "rag", "per_context", "tree"]
     dec_t = [0]                                                               # decode step counter, walks 0..255 and wraps
 
     def step(ev=None):
@@ -457,6 +468,7 @@ def main():
         leg("shared", lambda: plan_s.attend(db.T, db.S, ws_s))
         leg("rag", lambda: plan_g.attend(rb.T, rb.S, ws_g))
         leg("per_context", lambda: plan_pc.attend(pb.T, pb.S, ws_pc))
+        leg("tree", lambda: plan_t.attend(pb.T, pb.S, ws_t))
         for i in range(R):
             flush.zero_()
             if ev: ev["cfg2"][i][0].record()
@@ -592,13 +604,13 @@ def main():
     by_step0 = decode_bytes(DEC_REQ, dec_tokens(0))
     cpu = None if args.no_cpu_baseline else cpu_oracle_sample()
     n_launch = R * (3 + plan_e.last_launches() + plan_p.last_launches() + plan_d.last_launches() + plan_s.last_launches()
-                    + plan_g.last_launches() + plan_pc.last_launches() + plan_ce.last_launches() + plan_c.last_launches())
+                    + plan_g.last_launches() + plan_pc.last_launches() + plan_t.last_launches() + plan_ce.last_launches() + plan_c.last_launches())
     line = {
         "metric": METRIC, "value": world * tf_prefill, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "reps_per_step": R, "ms_per_step": t["step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "statistic": "median over steps of (leg time / reps_per_step); ms_per_step is the mean",
         "config": {"workload": "cfg4_manyshot_128k prefill (value) + cfg5 decode x16 + rope/encode 500x256, Llama-3-8B head shape; "
-                               "also timed: cfg3 RAG prefill, cfg2 encode + prefill, per-context form",
+                               "also timed: cfg3 RAG prefill, cfg2 encode + prefill, per-context and tree forms",
                    "H_q": H_Q, "H_kv": H_KV, "d": D, "prefix": L_P, "contexts": f"{N_CTX}x{L_CTX}", "query_rows": L_Q,
                    "decode_batch": DEC_REQ, "T": pb.T, "S": pb.S,
                    "l2": "inputs larger than L2 (0.53 GB / 8.4 GB / 0.34 GB KV per pass); cfg2 fits L2 and is flushed (256 MB write) before every repetition",
@@ -621,6 +633,8 @@ def main():
         "rag_cfg3": tensor_leg(t["rag"], fl_rag),
         "cfg2": {"encode": tensor_leg(t["c2_enc"], fl_c2_enc), "prefill": tensor_leg(t["c2_pre"], fl_c2_pre), "l2": "flushed before every repetition"},
         "per_context_form": dict(tensor_leg(t["per_context"], fl_prefill), what="the 128K prefill planned with ape_attend_plan_per_context (Eq. 11-12)"),
+        "tree_form": dict(tensor_leg(t["tree"], fl_prefill), what="the 128K prefill over a two-level context tree, 50 documents x 10 chunks, "
+                          "S per document (ape_attend_plan_tree)"),
         "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": args.steps * n_launch,
         "wall_s_timed_region": t_wall,

@@ -122,6 +122,27 @@ int ape_attend_plan_per_context(ape_handle_t handle, const ape_shape_t *shape, c
                                 const ape_request_t *requests, int32_t n_req, ape_mode_t mode, ape_plan_t *plan);
 
 /*
+ * Same as ape_attend_plan, for contexts that form trees (appendix "Future Directions": each context a tree-like
+ * hierarchy, evaluated along each branch with intermediate results merged on the way; built on the appendix
+ * "Hierarchical Formula for APE", Eq. 11-12).  requests[r].ctx[i] is node i of request r: its own tokens (the span may be
+ * empty: a node that only groups its children); parent[r][i] is its parent node, -1 for a top-level node, and
+ * parent[r][i] < i (children are listed after their parent).  At most 16 levels.
+ * Evaluation, per query row: inside a node its members -- its own tokens (logits divided by T) and its finished child
+ * nodes -- merge by the plain hierarchical softmax identity into the node's output V_n and log-sum-exp A_n; a node with
+ * scaled[r][i] != 0 enters its parent's merge with S * A_n (the A^{h'} = S * LogSumExp of Eq. 11), the others with A_n;
+ * the top-level nodes and the non-context segment meet in the final softmax.  `scaled` (or scaled[r]) may be NULL: then
+ * exactly the top-level nodes are scaled, i.e. every top-level tree is one context of Eq. 11-12.  Two ends of this
+ * family are printed formulas: one node per context gives Eq. 11-12 (ape_attend_plan_per_context), one tree over all
+ * contexts gives Eq. 5 (ape_attend_plan).  The paper prints no formula for deeper hierarchies; where S applies along a
+ * branch is this library's reading, made explicit by `scaled`.
+ * Launch with ape_attend.  Work items are cut at node boundaries.  APE_ERR_INVALID_ARG for a malformed tree.
+ */
+int ape_attend_plan_tree(ape_handle_t handle, const ape_shape_t *shape, const ape_kv_pool_t *pool,
+                         const ape_rows_t *q, const ape_rows_t *out, float *lse,
+                         const ape_request_t *requests, int32_t n_req,
+                         const int32_t *const *parent, const uint8_t *const *scaled, ape_mode_t mode, ape_plan_t *plan);
+
+/*
  * Decode for a batch of requests that attend to the SAME cached contexts (the serving case the paper's cache argument
  * describes: many queries over one set of pre-encoded documents or shots; section "Parallel Encoding", pre-caching).
  * Every request has q_len 1, its row of Q directly follows the previous request's (q_start = requests[0].q_start + r),
@@ -241,7 +262,7 @@ int ape_decode_noalloc(const ape_shape_t *shape, const ape_kv_pool_t *pool, cons
  * "Hierarchical Formula for Softmax Attention"), applies the scaling factor S to the combined context LSE and merges with
  * the non-context segment (Eq. 5).  The result equals ape_attend over all contexts.  All four arrays are DEVICE, fp32,
  * caller-owned: o_* [q rows, H_q, d], lse_* [q rows, H_q], indexed like Q; a segment without keys has lse = -inf.
- * Not available for per-context plans (APE_ERR_MODE).
+ * Not available for per-context and tree plans (APE_ERR_MODE).
  */
 typedef struct { float *o_ctx, *lse_ctx, *o_oth, *lse_oth; } ape_partials_t;
 

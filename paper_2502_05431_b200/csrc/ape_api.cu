@@ -57,7 +57,8 @@ struct ape_plan_s {
     int split_r = 0;
     bool o_via_tma = false;         // encode plans: tm_o describes the output rows
     int32_t last_launches = 0;
-    bool per_context = false;        // merge form: Eq. 5 (false) or Eq. 11-12 (true)
+    int per_context = 0;             // merge form: 0 Eq. 5, 1 Eq. 11-12 (per context), 2 context trees
+    DevNode* d_nodes = nullptr;      // tree plans
     // shared-context decode plans: the context pass of all requests (tensor-core kernel) and the per-request rest (decode kernel)
     ape_plan_s* child_ctx = nullptr;
     ape_plan_s* child_oth = nullptr;
@@ -156,20 +157,43 @@ std::vector<ape_span_t> fuse_spans(const ape_span_t* ctx, int n) {
 }
 
 // Tile ranges of the context segment: one range over the fused spans (Eq. 5 form), or one range per non-empty
-// context in the caller's order (per-context form).
-std::vector<std::pair<int, int>> add_context_tiles(std::vector<DevTile>& tiles, const ape_span_t* ctx, int n, int tile, bool per_context) {
-    std::vector<std::pair<int, int>> ranges;
+// context in the caller's order (per-context form; `id` is the context's ordinal among the non-empty ones).
+struct CtxRange { int t0, t1, id; };
+std::vector<CtxRange> add_context_tiles(std::vector<DevTile>& tiles, const ape_span_t* ctx, int n, int tile, bool per_context) {
+    std::vector<CtxRange> ranges;
     if (!per_context) {
         const int t0 = static_cast<int>(tiles.size());
         for (const auto& s : fuse_spans(ctx, n)) add_span_tiles(tiles, s.start, s.len, tile, 0, 0);
-        if (static_cast<int>(tiles.size()) > t0) ranges.push_back({t0, static_cast<int>(tiles.size())});
+        if (static_cast<int>(tiles.size()) > t0) ranges.push_back({t0, static_cast<int>(tiles.size()), 0});
     } else {
         for (int i = 0; i < n; ++i) {
             if (ctx[i].len <= 0) continue;
             const int t0 = static_cast<int>(tiles.size());
             add_span_tiles(tiles, ctx[i].start, ctx[i].len, tile, 0, 0);
-            ranges.push_back({t0, static_cast<int>(tiles.size())});
+            ranges.push_back({t0, static_cast<int>(tiles.size()), static_cast<int>(ranges.size())});
         }
+    }
+    return ranges;
+}
+
+// Context trees: the nodes of one request in depth-first order (a node's own tokens, then its subtrees, children in
+// index order), one tile range per node that holds tokens; `id` is the node's index in the plan-wide node array.  The
+// merge kernel relies on this order: once the walk has left a subtree it never returns to it.
+std::vector<CtxRange> add_tree_tiles(std::vector<DevTile>& tiles, const ape_span_t* ctx, const int32_t* parent, int n, int tile,
+                                     int node_base) {
+    std::vector<std::vector<int>> children(n);
+    std::vector<int> roots, stack;
+    for (int i = 0; i < n; ++i) (parent[i] < 0 ? roots : children[parent[i]]).push_back(i);
+    std::vector<CtxRange> ranges;
+    for (auto r = roots.rbegin(); r != roots.rend(); ++r) stack.push_back(*r);
+    while (!stack.empty()) {
+        const int i = stack.back(); stack.pop_back();
+        if (ctx[i].len > 0) {
+            const int t0 = static_cast<int>(tiles.size());
+            add_span_tiles(tiles, ctx[i].start, ctx[i].len, tile, 0, 0);
+            ranges.push_back({t0, static_cast<int>(tiles.size()), node_base + i});
+        }
+        for (auto c = children[i].rbegin(); c != children[i].rend(); ++c) stack.push_back(*c);
     }
     return ranges;
 }
@@ -180,6 +204,7 @@ struct HostMeta {
     std::vector<int32_t> cta_begin;
     std::vector<DevReq> reqs;
     std::vector<DevMerge> merge;
+    std::vector<DevNode> nodes;      // tree plans
 };
 
 struct Run {   // a run of tiles of one segment for one (request, kv head, row-block group)
@@ -233,8 +258,8 @@ int upload(ape_plan_t p, const HostMeta& m) {
     auto rnd = [](size_t x) { return (x + 255) & ~size_t(255); };
     const size_t b_tiles = rnd(m.tiles.size() * sizeof(DevTile) + 16), b_items = rnd(m.items.size() * sizeof(DevItem) + 16),
                  b_cta = rnd(m.cta_begin.size() * 4 + 16), b_reqs = rnd(m.reqs.size() * sizeof(DevReq) + 16),
-                 b_merge = rnd(m.merge.size() * sizeof(DevMerge) + 16);
-    const size_t total = b_tiles + b_items + b_cta + b_reqs + b_merge;
+                 b_merge = rnd(m.merge.size() * sizeof(DevMerge) + 16), b_nodes = rnd(m.nodes.size() * sizeof(DevNode) + 16);
+    const size_t total = b_tiles + b_items + b_cta + b_reqs + b_merge + b_nodes;
     std::vector<uint8_t> host(total, 0);
     size_t o = 0;
     auto put = [&](const void* src, size_t n, size_t padded) { if (n) std::memcpy(host.data() + o, src, n); size_t at = o; o += padded; return at; };
@@ -243,6 +268,7 @@ int upload(ape_plan_t p, const HostMeta& m) {
     const size_t o_cta = put(m.cta_begin.data(), m.cta_begin.size() * 4, b_cta);
     const size_t o_reqs = put(m.reqs.data(), m.reqs.size() * sizeof(DevReq), b_reqs);
     const size_t o_merge = put(m.merge.data(), m.merge.size() * sizeof(DevMerge), b_merge);
+    const size_t o_nodes = put(m.nodes.data(), m.nodes.size() * sizeof(DevNode), b_nodes);
     if (cudaMalloc(&p->d_blob, total) != cudaSuccess) { p->d_blob = nullptr; return APE_ERR_NOMEM; }
     if (cudaMemcpy(p->d_blob, host.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) return APE_ERR_CUDA;
     uint8_t* b = static_cast<uint8_t*>(p->d_blob);
@@ -251,6 +277,7 @@ int upload(ape_plan_t p, const HostMeta& m) {
     p->d_cta_begin = reinterpret_cast<int32_t*>(b + o_cta);
     p->d_reqs = reinterpret_cast<DevReq*>(b + o_reqs);
     p->d_merge = reinterpret_cast<DevMerge*>(b + o_merge);
+    p->d_nodes = reinterpret_cast<DevNode*>(b + o_nodes);
     p->n_items = static_cast<int>(m.items.size());
     p->n_merge = static_cast<int>(m.merge.size());
     return APE_OK;
@@ -339,7 +366,7 @@ int ape_plan_destroy(ape_plan_t p) {
 
 static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
                             const ape_rows_t* out, float* lse, const ape_request_t* reqs, int32_t n_req, ape_mode_t mode,
-                            bool per_context, ape_plan_t* plan_out)
+                            int per_context, const int32_t* const* parent, const uint8_t* const* scaled, ape_plan_t* plan_out)
 {
     if (!h || !plan_out) return APE_ERR_INVALID_ARG;
     *plan_out = nullptr;
@@ -364,6 +391,32 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
         if (rq.query_kv_capacity < rq.query_kv.len || rq.query_kv.start + rq.query_kv_capacity > pool->n_tokens) return APE_ERR_INVALID_ARG;
         max_extra = std::min(max_extra, rq.query_kv_capacity - rq.query_kv.len);
     }
+    HostMeta m;
+    std::vector<int> node_base(n_req, 0);
+    if (per_context == 2) {
+        // the trees: parent[i] < i keeps them acyclic; depth is bounded by what the merge kernel's stack holds
+        if (!parent) return APE_ERR_INVALID_ARG;
+        try {
+            for (int r = 0; r < n_req; ++r) {
+                const int n = reqs[r].n_ctx;
+                if (n > 0 && !parent[r]) return APE_ERR_INVALID_ARG;
+                node_base[r] = static_cast<int>(m.nodes.size());
+                for (int i = 0; i < n; ++i) {
+                    const int par = parent[r][i];
+                    if (par < -1 || par >= i) return APE_ERR_INVALID_ARG;
+                    DevNode nd;
+                    nd.parent = par < 0 ? -1 : node_base[r] + par;
+                    nd.depth = par < 0 ? 0 : m.nodes[node_base[r] + par].depth + 1;
+                    if (nd.depth >= kMaxTreeDepth) return APE_ERR_INVALID_ARG;
+                    nd.scaled = (scaled && scaled[r]) ? (scaled[r][i] ? 1 : 0) : (par < 0 ? 1 : 0);
+                    nd.pad = 0;
+                    m.nodes.push_back(nd);
+                }
+            }
+        } catch (const std::bad_alloc&) {
+            return APE_ERR_NOMEM;
+        }
+    }
     DeviceGuard guard(h->device);
     if (!guard.ok) return APE_ERR_CUDA;
 
@@ -374,7 +427,6 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
     p->max_kv_extra = (mode == APE_DECODE) ? max_extra : 0;
     const int D = shape->head_dim, H_kv = shape->n_kv_heads;
 
-    HostMeta m;
     std::vector<Run> runs;
     try {
         if (mode == APE_DECODE) {
@@ -389,14 +441,15 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
                 add_span_tiles(m.tiles, rq.prefix.start, rq.prefix.len, tile, 0, 0);
                 add_span_tiles(m.tiles, rq.query_kv.start, rq.query_kv.len, tile, TILE_GROWS, rq.query_kv_capacity);
                 const int o1 = static_cast<int>(m.tiles.size());
-                const auto ctx_ranges = add_context_tiles(m.tiles, rq.ctx, rq.n_ctx, tile, per_context);
+                const auto ctx_ranges = (per_context == 2) ? add_tree_tiles(m.tiles, rq.ctx, parent[r], rq.n_ctx, tile, node_base[r])
+                                                            : add_context_tiles(m.tiles, rq.ctx, rq.n_ctx, tile, per_context == 1);
                 for (int hh = 0; hh < H_kv; ++hh) {
                     DevMerge g{r, hh, 0, 0, 0, 0, 0, 1};
                     const int mi = static_cast<int>(m.merge.size());
                     m.merge.push_back(g);
                     runs.push_back(Run{r, hh, 0, 1, SEG_OTHER, o0, o1, mi});
                     for (size_t ci = 0; ci < ctx_ranges.size(); ++ci)
-                        runs.push_back(Run{r, hh, 0, 1, SEG_CTX, ctx_ranges[ci].first, ctx_ranges[ci].second, mi, static_cast<int>(ci)});
+                        runs.push_back(Run{r, hh, 0, 1, SEG_CTX, ctx_ranges[ci].t0, ctx_ranges[ci].t1, mi, ctx_ranges[ci].id});
                 }
             }
             p->n_cta = h->n_sm;
@@ -426,7 +479,8 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
                 add_span_tiles(m.tiles, rq.prefix.start, rq.prefix.len, tile, 0, 0);
                 add_span_tiles(m.tiles, rq.query_kv.start, rq.query_kv.len, tile, TILE_CAUSAL, 0);
                 const int o1 = static_cast<int>(m.tiles.size());
-                const auto ctx_ranges = add_context_tiles(m.tiles, rq.ctx, rq.n_ctx, tile, per_context);
+                const auto ctx_ranges = (per_context == 2) ? add_tree_tiles(m.tiles, rq.ctx, parent[r], rq.n_ctx, tile, node_base[r])
+                                                            : add_context_tiles(m.tiles, rq.ctx, rq.n_ctx, tile, per_context == 1);
                 const int RB = static_cast<int>((rq.q_len + TB - 1) / TB);
                 for (int hh = 0; hh < H_kv; ++hh) {
                     for (int rb0 = 0; rb0 < RB; rb0 += p->n_sib) {
@@ -435,7 +489,7 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
                         for (int s = 0; s < live; ++s) m.merge.push_back(DevMerge{r, hh, rb0 + s, 0, 0, 0, 0, 1});
                         runs.push_back(Run{r, hh, rb0, live, SEG_OTHER, o0, o1, mi});
                         for (size_t ci = 0; ci < ctx_ranges.size(); ++ci)
-                            runs.push_back(Run{r, hh, rb0, live, SEG_CTX, ctx_ranges[ci].first, ctx_ranges[ci].second, mi, static_cast<int>(ci)});
+                            runs.push_back(Run{r, hh, rb0, live, SEG_CTX, ctx_ranges[ci].t0, ctx_ranges[ci].t1, mi, ctx_ranges[ci].id});
                     }
                 }
             }
@@ -463,14 +517,21 @@ int ape_attend_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
                     const ape_rows_t* out, float* lse, const ape_request_t* reqs, int32_t n_req, ape_mode_t mode,
                     ape_plan_t* plan_out)
 {
-    return attend_plan_impl(h, shape, pool, q, out, lse, reqs, n_req, mode, false, plan_out);
+    return attend_plan_impl(h, shape, pool, q, out, lse, reqs, n_req, mode, 0, nullptr, nullptr, plan_out);
 }
 
 int ape_attend_plan_per_context(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
                                 const ape_rows_t* out, float* lse, const ape_request_t* reqs, int32_t n_req, ape_mode_t mode,
                                 ape_plan_t* plan_out)
 {
-    return attend_plan_impl(h, shape, pool, q, out, lse, reqs, n_req, mode, true, plan_out);
+    return attend_plan_impl(h, shape, pool, q, out, lse, reqs, n_req, mode, 1, nullptr, nullptr, plan_out);
+}
+
+int ape_attend_plan_tree(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
+                         const ape_rows_t* out, float* lse, const ape_request_t* reqs, int32_t n_req,
+                         const int32_t* const* parent, const uint8_t* const* scaled, ape_mode_t mode, ape_plan_t* plan_out)
+{
+    return attend_plan_impl(h, shape, pool, q, out, lse, reqs, n_req, mode, 2, parent, scaled, plan_out);
 }
 
 int ape_attend_plan_shared(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
@@ -866,7 +927,7 @@ static int attend_impl(ape_plan_t p, float T, float S, int64_t kv_extra, void* w
         if (launch_decode(D, b->tm_k, b->tm_v, dp, b->n_cta, b->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
         p->last_launches++;
         MergeParams mp;
-        mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.items = nullptr; mp.per_context = 0; mp.n_groups = p->n_merge;
+        mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.items = nullptr; mp.per_context = 0; mp.nodes = nullptr; mp.n_groups = p->n_merge;
         mp.rows_per_slot = G; mp.tokens_per_block = 1; mp.ws_o = b_o; mp.ws_ml = b_ml;
         mp.ws_o_ctx = a_o; mp.ws_ml_ctx = a_ml; mp.rows_per_slot_ctx = kAttnRows;
         mp.out = rows_desc(p->out); mp.lse_out = p->lse; mp.S = S; mp.G = G; mp.H_q = p->shape.n_q_heads; mp.D = D;
@@ -901,7 +962,7 @@ static int attend_impl(ape_plan_t p, float T, float S, int64_t kv_extra, void* w
     p->last_launches++;
 
     MergeParams mp;
-    mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.items = p->d_items; mp.per_context = p->per_context ? 1 : 0; mp.n_groups = p->n_merge; mp.rows_per_slot = rows_per_slot;
+    mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.items = p->d_items; mp.per_context = p->per_context; mp.nodes = p->d_nodes; mp.n_groups = p->n_merge; mp.rows_per_slot = rows_per_slot;
     mp.tokens_per_block = rows_per_slot / G; mp.ws_o = ws_o; mp.ws_ml = ws_ml; mp.out = rows_desc(p->out); mp.lse_out = p->lse;
     mp.ws_o_ctx = ws_o; mp.ws_ml_ctx = ws_ml; mp.rows_per_slot_ctx = rows_per_slot;
     mp.S = S; mp.G = G; mp.H_q = p->shape.n_q_heads; mp.D = D;
@@ -1234,7 +1295,7 @@ int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, cons
                 const int mi = static_cast<int>(m.merge.size());
                 m.merge.push_back(DevMerge{r, hh, 0, 0, 0, 0, 0, 1});
                 runs.push_back(Run{r, hh, 0, 1, SEG_OTHER, o0, o1, mi});
-                for (const auto& cr : ctx_ranges) runs.push_back(Run{r, hh, 0, 1, SEG_CTX, cr.first, cr.second, mi});
+                for (const auto& cr : ctx_ranges) runs.push_back(Run{r, hh, 0, 1, SEG_CTX, cr.t0, cr.t1, mi});
             }
         }
         assign_stream(runs, n_cta, 1, m);
@@ -1290,7 +1351,7 @@ int ape_decode_noalloc(const ape_shape_t* shape, const ape_kv_pool_t* pool, cons
     dp.kv_extra = static_cast<int32_t>(kv_extra); dp.G = G; dp.n_stages = n_stages; dp.status = reinterpret_cast<int*>(base);
     if (launch_decode(D, tm_k, tm_v, dp, n_cta, smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
     MergeParams mp;
-    mp.groups = reinterpret_cast<const DevMerge*>(base + o_merge); mp.reqs = dp.reqs; mp.items = dp.items; mp.per_context = 0; mp.n_groups = static_cast<int32_t>(m.merge.size());
+    mp.groups = reinterpret_cast<const DevMerge*>(base + o_merge); mp.reqs = dp.reqs; mp.items = dp.items; mp.per_context = 0; mp.nodes = nullptr; mp.n_groups = static_cast<int32_t>(m.merge.size());
     mp.rows_per_slot = G; mp.tokens_per_block = 1; mp.ws_o = ws_o; mp.ws_ml = ws_ml; mp.out = rows_desc(*out); mp.lse_out = lse;
     mp.ws_o_ctx = ws_o; mp.ws_ml_ctx = ws_ml; mp.rows_per_slot_ctx = G;
     mp.part_o_ctx = nullptr; mp.part_lse_ctx = nullptr; mp.part_o_oth = nullptr; mp.part_lse_oth = nullptr;

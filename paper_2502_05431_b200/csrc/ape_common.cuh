@@ -37,7 +37,8 @@ struct DevItem {
     int32_t q_row0;      // first row of Q / O of the request (encode: context start)
     int32_t q_len;       // query rows of the request
     int32_t l_k;         // keys in the query segment at planning time (encode: context length)
-    int32_t ctx_id;      // SEG_CTX items of a per-context plan: ordinal of the context the tiles belong to, else 0
+    int32_t ctx_id;      // SEG_CTX items: ordinal of the context (per-context plans) or index of the tree node (tree plans)
+                         // the tiles belong to, else 0
     DevTile first_tile;  // tiles[tile_begin]
 };
 static_assert(sizeof(DevItem) == 64, "DevItem is one 64-byte record");
@@ -65,6 +66,15 @@ struct DevMerge {
                          // partials of many requests in one slot, one group of rows per request
     int32_t ctx_stride;  // between consecutive context partials
 };
+
+// One node of a context tree (tree plans): a SEG_CTX item's ctx_id is the index of the node its tiles belong to.
+struct DevNode {
+    int32_t parent;      // index of the parent node in the same array, -1 for a top-level node
+    int32_t depth;       // 0 for a top-level node
+    int32_t scaled;      // != 0: the node hands S * log-sum-exp to its parent (Eq. 11), else its plain log-sum-exp
+    int32_t pad;
+};
+constexpr int kMaxTreeDepth = 16;   // levels of nodes below the final merge
 
 struct RowsDesc {        // Q or O rows: element (r, h, e) at data[r*token_stride + h*head_stride + e]
     __nv_bfloat16* data;

@@ -66,7 +66,9 @@ struct MergeParams {
     const DevMerge* groups;
     const DevReq* reqs;
     const DevItem* items;            // per-context mode: the context ordinal of a partial is items[slot / slot_stride].ctx_id
-    int32_t per_context;             // 0: Eq. 5 (S on the LSE of all contexts together); 1: Eq. 11-12 (S on every context's own LSE)
+    int32_t per_context;             // 0: Eq. 5 (S on the LSE of all contexts together); 1: Eq. 11-12 (S on every context's own LSE);
+                                     // 2: context trees (the hierarchical formula node by node, S where a node is marked)
+    const DevNode* nodes;            // tree plans: all requests' nodes
     int32_t n_groups;
     int32_t rows_per_slot;           // G (decode) or kAttnRows (prefill)
     int32_t tokens_per_block;        // query tokens per row block: rows_per_slot / G

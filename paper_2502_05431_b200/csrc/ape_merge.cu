@@ -91,6 +91,75 @@ __device__ __forceinline__ void combine_per_context(const MergeParams& p, const 
     lse = (Z > 0.f) ? top + fast_log2(Z) : -INFINITY;
 }
 
+// Context trees (appendix "Future Directions" on top of "Hierarchical Formula for APE"): the partials of a row arrive in
+// depth-first order of the nodes their tiles belong to (a node's own tokens, then its subtrees).  A stack of accumulators,
+// one per open tree level, follows that order: a partial is added to its node's accumulator; when the walk leaves a node,
+// the node is finished -- log-sum-exp A_n and normalised output V_n of its members, by the plain hierarchical softmax
+// identity -- and handed to its parent's accumulator as one member with log weight S * A_n if the node is marked, A_n
+// otherwise.  Level 0 collects the top-level nodes; its content is the context side of the final softmax.
+template <int VEC>
+__device__ __forceinline__ void combine_tree(const MergeParams& p, const DevMerge& g, int row, int lane,
+                                             float& lse, float& norm, float (&acc)[VEC])
+{
+    float top[kMaxTreeDepth + 1], Z[kMaxTreeDepth + 1], a[kMaxTreeDepth + 1][VEC];
+    int node_at[kMaxTreeDepth + 1];
+    top[0] = -INFINITY; Z[0] = 0.f; node_at[0] = -1;
+    #pragma unroll
+    for (int v = 0; v < VEC; ++v) a[0][v] = 0.f;
+    int sp = 0;                                       // deepest open level; level k + 1 holds an open node of depth k
+    auto add = [&](int lv, float m, float l, const float (&o)[VEC]) {
+        const float Mn = fmaxf(top[lv], m);
+        const float f_old = fast_exp2(top[lv] - Mn), f_new = fast_exp2(m - Mn);
+        #pragma unroll
+        for (int v = 0; v < VEC; ++v) a[lv][v] = a[lv][v] * f_old + o[v] * f_new;
+        Z[lv] = Z[lv] * f_old + l * f_new;
+        top[lv] = Mn;
+    };
+    auto close = [&](int lv) {                        // finish the node at level lv and hand it to level lv - 1
+        if (Z[lv] > 0.f) {
+            const float A = top[lv] + fast_log2(Z[lv]);
+            const float handed = p.nodes[node_at[lv]].scaled ? p.S * A : A;
+            const float inv = 1.f / Z[lv];
+            float o[VEC];
+            #pragma unroll
+            for (int v = 0; v < VEC; ++v) o[v] = a[lv][v] * inv;
+            add(lv - 1, handed, 1.f, o);
+        }
+    };
+    auto ancestor = [&](int node, int depth_now, int depth_want) {
+        for (; depth_now > depth_want; --depth_now) node = p.nodes[node].parent;
+        return node;
+    };
+    const int item0 = g.ctx_slot0 / g.slot_stride;
+    for (int i = 0; i < g.ctx_n; ++i) {
+        const int node = p.items[item0 + i].ctx_id;
+        const int depth = p.nodes[node].depth;
+        // leave every open node that is not on the path from the top level down to `node`
+        while (sp > 0 && (sp - 1 > depth || ancestor(node, depth, sp - 1) != node_at[sp])) { close(sp); --sp; }
+        // open the rest of that path
+        while (sp < depth + 1) {
+            ++sp;
+            node_at[sp] = ancestor(node, depth, sp - 1);
+            top[sp] = -INFINITY; Z[sp] = 0.f;
+            #pragma unroll
+            for (int v = 0; v < VEC; ++v) a[sp][v] = 0.f;
+        }
+        const size_t slot = static_cast<size_t>(g.ctx_slot0) + static_cast<size_t>(i) * g.slot_stride;
+        const float2 ml = *reinterpret_cast<const float2*>(p.ws_ml + (slot * p.rows_per_slot + row) * 2);
+        if (!(ml.y > 0.f)) continue;
+        const float* src = p.ws_o + (slot * p.rows_per_slot + row) * p.D + lane * VEC;
+        float x[VEC];
+        if constexpr (VEC == 4) { const float4 t = *reinterpret_cast<const float4*>(src); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
+        else { const float2 t = *reinterpret_cast<const float2*>(src); x[0] = t.x; x[1] = t.y; }
+        add(sp, ml.x, ml.y, x);
+    }
+    while (sp > 0) { close(sp); --sp; }
+    #pragma unroll
+    for (int v = 0; v < VEC; ++v) acc[v] = a[0][v];
+    norm = Z[0];
+    lse = (Z[0] > 0.f) ? top[0] + fast_log2(Z[0]) : -INFINITY;
+}
+
 template <int VEC>
 __global__ void __launch_bounds__(256) ape_merge_kernel(const MergeParams p)
 {
@@ -107,7 +176,9 @@ __global__ void __launch_bounds__(256) ape_merge_kernel(const MergeParams p)
 
     float Mc, Lc, Mo, Lo, ac[VEC], ao[VEC];
     float lse_c;
-    if (p.per_context) {
+    if (p.per_context == 2) {
+        combine_tree<VEC>(p, g, row, lane, lse_c, Lc, ac);             // Lc: the normaliser of ac
+    } else if (p.per_context == 1) {
         combine_per_context<VEC>(p, g, row, lane, lse_c, Lc, ac);      // Lc: the normaliser of ac
     } else {
         combine_segment<VEC>(p.ws_o_ctx, p.ws_ml_ctx, g.ctx_slot0, g.ctx_n, g.ctx_stride, p.rows_per_slot_ctx, row + g.ctx_row_off,

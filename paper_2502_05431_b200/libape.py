@@ -22,7 +22,7 @@ EXPORTS = ["ape_create", "ape_destroy", "ape_attend_plan", "ape_encode_plan", "a
            "ape_get_status", "ape_status_string", "ape_decode_noalloc", "ape_attend_plan_per_context",
            "ape_rope_runs_for_request", "ape_rope_plan", "ape_rope_write", "ape_attend_plan_shared",
            "ape_attend_partial", "ape_merge_shards", "ape_selftest_timeout", "ape_selftest_timeout_noalloc",
-           "ape_set_sm_budget", "ape_get_status_stream", "ape_decode_step_host"]
+           "ape_set_sm_budget", "ape_get_status_stream", "ape_decode_step_host", "ape_attend_plan_tree"]
 
 
 class ApeError(RuntimeError):
@@ -78,6 +78,8 @@ def load() -> C.CDLL:
                                         C.POINTER(ape_rows_t), vp, C.POINTER(ape_request_t), C.c_int32, C.c_int, C.POINTER(vp)]
         lib.ape_attend_plan_per_context.argtypes = lib.ape_attend_plan.argtypes
         lib.ape_attend_plan_shared.argtypes = lib.ape_attend_plan.argtypes[:7] + lib.ape_attend_plan.argtypes[8:]
+        lib.ape_attend_plan_tree.argtypes = lib.ape_attend_plan.argtypes[:8] + [C.POINTER(C.POINTER(C.c_int32)),
+                                                                                C.POINTER(C.POINTER(C.c_uint8)), C.c_int, C.POINTER(vp)]
         lib.ape_encode_plan.argtypes = [vp, C.POINTER(ape_shape_t), C.POINTER(ape_kv_pool_t), C.POINTER(ape_rows_t),
                                         C.POINTER(ape_rows_t), vp, C.POINTER(ape_span_t), C.POINTER(ape_span_t), C.c_int32,
                                         C.POINTER(vp)]
@@ -213,10 +215,12 @@ class Handle:
     def attend_plan(self, *, H_q: int, H_kv: int, d: int, k_pool: torch.Tensor, v_pool: torch.Tensor,
                     q: torch.Tensor, out: torch.Tensor, requests: Sequence, mode: int,
                     lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0, per_context: bool = False,
-                    shared: bool = False) -> "Plan":
+                    shared: bool = False, tree=None) -> "Plan":
         """ape_attend_plan (or ape_attend_plan_per_context: S on every context's own LSE, Eq. 11-12; or, with shared=True,
         ape_attend_plan_shared: a decode batch whose requests all attend to the same contexts).  `requests`: objects with q_start, q_len, prefix, ctx, query_kv, query_kv_capacity
-        (spans are (start, len) pairs), e.g. paper_2502_05431_b200.workloads.Request."""
+        (spans are (start, len) pairs), e.g. paper_2502_05431_b200.workloads.Request.
+        `tree` = (parents, scaled) selects ape_attend_plan_tree: parents[r][i] is the parent of request r's node i (its
+        ctx[i]), -1 at the top level; scaled (or scaled[r]) may be None (the top-level nodes carry S)."""
         shape = ape_shape_t(H_q, H_kv, d, softmax_scale)
         pool, qr, orows = _pool(k_pool, v_pool), _rows(q), _rows(out)
         n = len(requests)
@@ -228,6 +232,19 @@ class Handle:
             arr[i] = ape_request_t(int(r.q_start), int(r.q_len), ape_span_t(*map(int, r.prefix)), spans, len(r.ctx),
                                    ape_span_t(*map(int, r.query_kv)), int(r.query_kv_capacity))
         p = C.c_void_p()
+        if tree is not None:
+            parents, scaled = tree
+            par_arrs = [(C.c_int32 * max(len(pp), 1))(*[int(x) for x in pp]) for pp in parents]
+            par = (C.POINTER(C.c_int32) * max(n, 1))(*[C.cast(a, C.POINTER(C.c_int32)) for a in par_arrs])
+            sc = None
+            if scaled is not None:
+                sc_arrs = [None if ss is None else (C.c_uint8 * max(len(ss), 1))(*[1 if x else 0 for x in ss]) for ss in scaled]
+                sc = (C.POINTER(C.c_uint8) * max(n, 1))(*[C.cast(a, C.POINTER(C.c_uint8)) if a is not None
+                                                         else C.POINTER(C.c_uint8)() for a in sc_arrs])
+            _check(load().ape_attend_plan_tree(self._h, C.byref(shape), C.byref(pool), C.byref(qr), C.byref(orows),
+                                               lse.data_ptr() if lse is not None else None, arr, n, par, sc, int(mode), C.byref(p)),
+                   "ape_attend_plan_tree")
+            return Plan(self, p, (q, out, k_pool, v_pool, lse))
         if shared:
             _check(load().ape_attend_plan_shared(self._h, C.byref(shape), C.byref(pool), C.byref(qr), C.byref(orows),
                                                  lse.data_ptr() if lse is not None else None, arr, n, C.byref(p)),

@@ -22,7 +22,7 @@ def handle() -> libape.Handle:
 
 
 def gpu_attend(b: Batch, mode: int, *, kv_extra: int = 0, want_lse: bool = True, q_override=None, per_context: bool = False,
-               shared: bool = False):
+               shared: bool = False, tree=None):
     """Copy the batch to cuda:0, plan, launch, return (out bf16 CPU, lse fp32 CPU, plan launches)."""
     dev = torch.device("cuda:0")
     q = (b.q if q_override is None else q_override).to(dev)
@@ -30,7 +30,7 @@ def gpu_attend(b: Batch, mode: int, *, kv_extra: int = 0, want_lse: bool = True,
     out = torch.full_like(q, float("nan"))
     lse = torch.full((q.shape[0], b.H_q), float("nan"), dtype=torch.float32, device=dev) if want_lse else None
     plan = handle().attend_plan(H_q=b.H_q, H_kv=b.H_kv, d=b.d, k_pool=k, v_pool=v, q=q, out=out,
-                                requests=b.requests, mode=mode, lse=lse, per_context=per_context, shared=shared)
+                                requests=b.requests, mode=mode, lse=lse, per_context=per_context, shared=shared, tree=tree)
     ws, check_bands = guarded_workspace(plan)
     plan.attend(b.T, b.S, ws, kv_extra=kv_extra)
     torch.cuda.synchronize()
