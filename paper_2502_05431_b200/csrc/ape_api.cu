@@ -56,6 +56,7 @@ struct ape_plan_s {
     SplitMaps tm_split{};           // encode plans with split_r > 0
     int split_r = 0;
     bool o_via_tma = false;         // encode plans: tm_o describes the output rows
+    bool alt_halves = false;        // context pass of a shared plan with at most 128 rows: the halves take alternate tiles
     int32_t last_launches = 0;
     int per_context = 0;             // merge form: 0 Eq. 5, 1 Eq. 11-12 (per context), 2 context trees
     DevNode* d_nodes = nullptr;      // tree plans
@@ -496,13 +497,13 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
             assign_stream(runs, n_groups, p->n_sib, m);
             p->n_cta = n_groups * p->n_sib;
             p->n_slots = static_cast<int>(m.items.size()) * p->n_sib;
-            p->smem_bytes = attn_smem_bytes(D, 1);
+            p->smem_bytes = attn_smem_bytes(D, 1, 0);
             const size_t rows = static_cast<size_t>(p->n_slots) * kAttnRows;
             p->ws_bytes = ((rows * D * 4 + 255) & ~size_t(255)) + ((rows * 2 * 4 + 255) & ~size_t(255));
             rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
             if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
             if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
-            if (!rc && attn_set_smem_attr(D, 1, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+            if (!rc && attn_set_smem_attr(D, 1, 0, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
         }
         if (!rc) { finish_items(m); rc = upload(p, m); }
     } catch (const std::bad_alloc&) {
@@ -586,7 +587,10 @@ int ape_attend_plan_shared(ape_handle_t h, const ape_shape_t* shape, const ape_k
         ape_plan_t a = p->child_ctx;
         HostMeta ma;
         std::vector<Run> runs_a;
-        const int TB = kAttnRows / G;
+        // With at most 128 query rows in the batch a 256-row block would be half empty: the row block then has 128 rows,
+        // both halves of a CTA hold them and take alternate tiles (two partials of 128 rows per slot).
+        a->alt_halves = n_req * G <= kAttnRows / 2;
+        const int TB = (a->alt_halves ? kAttnRows / 2 : kAttnRows) / G;
         const int RB = (n_req + TB - 1) / TB;
         a->n_sib = std::max(1, std::min({4, RB, h->n_sm}));
         const int n_groups = std::max(1, h->n_sm / a->n_sib);
@@ -604,11 +608,11 @@ int ape_attend_plan_shared(ape_handle_t h, const ape_shape_t* shape, const ape_k
         assign_stream(runs_a, n_groups, a->n_sib, ma);
         a->n_cta = n_groups * a->n_sib;
         a->n_slots = static_cast<int>(ma.items.size()) * a->n_sib;
-        a->smem_bytes = attn_smem_bytes(D, 1);
+        a->smem_bytes = attn_smem_bytes(D, 1, a->alt_halves ? 1 : 0);
         rc = make_map(h, &a->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, kAttnTileN);
         if (!rc) rc = make_map(h, &a->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, kAttnTileN);
         if (!rc) rc = make_map(h, &a->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
-        if (!rc && attn_set_smem_attr(D, 1, a->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+        if (!rc && attn_set_smem_attr(D, 1, a->alt_halves ? 1 : 0, a->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
         if (!rc) { finish_items(ma); rc = upload(a, ma); }
 
         // ---- the rest, per request: prefix + the request's own (growing) query segment ------------------------------
@@ -654,6 +658,11 @@ int ape_attend_plan_shared(ape_handle_t h, const ape_shape_t* shape, const ape_k
                     DevMerge g{r, hh, 0, ga.ctx_slot0, ga.ctx_n, gb.oth_slot0, gb.oth_n, std::max(1, gb.slot_stride)};
                     g.ctx_row_off = (r % TB) * G;
                     g.ctx_stride = ga.ctx_stride;
+                    if (a->alt_halves) {
+                        // one row block, one sibling: the items' slots are consecutive, and in units of 128 rows the two
+                        // partials of slot s are 2 s (half 0) and 2 s + 1 (half 1)
+                        g.ctx_slot0 = 2 * ga.ctx_slot0; g.ctx_n = 2 * ga.ctx_n; g.ctx_stride = 1;
+                    }
                     mp.merge.push_back(g);
                 }
             rc = upload(p, mp);
@@ -764,7 +773,7 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
         for (auto& b : bins) { for (auto& it : b) m.items.push_back(it); m.cta_begin.push_back(static_cast<int32_t>(m.items.size())); }
         p->n_slots = 0;
         p->ws_bytes = 0;
-        p->smem_bytes = attn_smem_bytes(D, 2);
+        p->smem_bytes = attn_smem_bytes(D, 2, 0);
         rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
         if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
         if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
@@ -777,7 +786,7 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
         // Every item of this plan has a row block of its own, so a finished row block may leave through its Q buffer.
         if (!rc) p->o_via_tma = make_map(h, &p->tm_o, out->data, D, shape->n_q_heads, out->n_rows, out->head_stride, out->token_stride,
                                          G, 128 / G) == APE_OK;
-        if (!rc && attn_set_smem_attr(D, 2, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+        if (!rc && attn_set_smem_attr(D, 2, 0, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
         if (!rc) { finish_items(m); rc = upload(p, m); }
     } catch (const std::bad_alloc&) {
         rc = APE_ERR_NOMEM;
@@ -915,7 +924,7 @@ static int attend_impl(ape_plan_t p, float T, float S, int64_t kv_extra, void* w
             ap.out = rows_desc(p->out); ap.lse_out = nullptr; ap.ws_o = a_o; ap.ws_ml = a_ml;
             ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c / T * kLog2e;
             ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = a->n_sib; ap.n_q_bufs = 1; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
-            ap.o_via_tma = 0; ap.split_r = 0;
+            ap.o_via_tma = 0; ap.split_r = 0; ap.alt_halves = a->alt_halves ? 1 : 0;
             if (launch_attn(D, a->tm_q, a->tm_k, a->tm_v, a->tm_q, a->tm_split, ap, a->n_cta, a->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
             p->last_launches++;
         }
@@ -929,7 +938,7 @@ static int attend_impl(ape_plan_t p, float T, float S, int64_t kv_extra, void* w
         MergeParams mp;
         mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.items = nullptr; mp.per_context = 0; mp.nodes = nullptr; mp.n_groups = p->n_merge;
         mp.rows_per_slot = G; mp.tokens_per_block = 1; mp.ws_o = b_o; mp.ws_ml = b_ml;
-        mp.ws_o_ctx = a_o; mp.ws_ml_ctx = a_ml; mp.rows_per_slot_ctx = kAttnRows;
+        mp.ws_o_ctx = a_o; mp.ws_ml_ctx = a_ml; mp.rows_per_slot_ctx = a->alt_halves ? kAttnRows / 2 : kAttnRows;
         mp.out = rows_desc(p->out); mp.lse_out = p->lse; mp.S = S; mp.G = G; mp.H_q = p->shape.n_q_heads; mp.D = D;
         mp.part_o_ctx = part ? part->o_ctx : nullptr; mp.part_lse_ctx = part ? part->lse_ctx : nullptr;
         mp.part_o_oth = part ? part->o_oth : nullptr; mp.part_lse_oth = part ? part->lse_oth : nullptr;
@@ -956,7 +965,7 @@ static int attend_impl(ape_plan_t p, float T, float S, int64_t kv_extra, void* w
         ap.out = rows_desc(p->out); ap.lse_out = nullptr; ap.ws_o = ws_o; ap.ws_ml = ws_ml;
         ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c / T * kLog2e;
         ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = p->n_sib; ap.n_q_bufs = 1; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
-        ap.o_via_tma = 0; ap.split_r = 0;
+        ap.o_via_tma = 0; ap.split_r = 0; ap.alt_halves = 0;
         if (launch_attn(D, p->tm_q, p->tm_k, p->tm_v, p->tm_q, p->tm_split, ap, p->n_cta, p->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
     }
     p->last_launches++;
@@ -1016,7 +1025,7 @@ int ape_encode_contexts(ape_plan_t p, void* workspace, size_t ws_bytes, void* st
     ap.out = rows_desc(p->out); ap.lse_out = p->lse; ap.ws_o = nullptr; ap.ws_ml = nullptr;
     ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c * kLog2e;
     ap.G = p->G; ap.H_q = p->shape.n_q_heads; ap.n_sib = 1; ap.n_q_bufs = 2; ap.q_rows_are_pool = 1; ap.status = p->h->d_status;
-    ap.o_via_tma = p->o_via_tma ? 1 : 0; ap.split_r = p->split_r;
+    ap.o_via_tma = p->o_via_tma ? 1 : 0; ap.split_r = p->split_r; ap.alt_halves = 0;
     if (launch_attn(p->shape.head_dim, p->tm_q, p->tm_k, p->tm_v, p->tm_o, p->tm_split, ap, p->n_cta, p->smem_bytes,
                     static_cast<cudaStream_t>(stream_v)) != cudaSuccess) return APE_ERR_CUDA;
     p->last_launches = 1;

@@ -15,6 +15,10 @@
 //   warp 11          with two Q buffers (encode): loads Q one row block ahead and hands finished O tiles to the bulk
 //                    tensor store; idle otherwise
 // The two halves run one tile apart, so that the tensor pipe works on one half while the other does its exponentials.
+// When a row block has at most 128 live rows (a decode batch that shares its contexts), the plan can ask for the
+// alternating form instead (ALT): both halves read the SAME 128 rows of Q and take every other tile, each with an online
+// softmax and a partial of its own, so no half works on rows that do not exist; the Q half that is not needed pays for a
+// third stage of K and of V, which a half that sees only every other tile needs to have its next tile under way.
 #include "ape_common.cuh"
 #include "ape_kernels.h"
 #include "ape_tcgen05.cuh"
@@ -30,7 +34,6 @@ constexpr int kRegsSoftmax = 216;            // registers per thread after the h
 constexpr int kRegsOther = 72;               // producer / MMA warpgroup
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
-constexpr int kNK = 2;                        // K stages
 constexpr int kSlabBytes = 128 * 128;         // 128 rows x 64 bf16
 constexpr float kRescaleThreshold = 8.0f;     // base-2 units: O is rescaled only when the row maximum grew by more
 constexpr float kLn2 = 0.6931471805599453f;
@@ -81,7 +84,7 @@ __device__ __forceinline__ bool tile_visible(const DevTile& t, const ItemGeom& g
 // QBUF: number of Q buffers.  Plans with long items (prefill) use one Q buffer and two stages each of K and V; plans
 // with many short items (encode) use two Q buffers, so that the next row block's Q arrives while the current one is
 // in use, and pay for them with a single V stage.
-template <int D, int QBUF>
+template <int D, int QBUF, bool ALT>
 __global__ void __launch_bounds__(kThreads, 1)
 ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -89,8 +92,10 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 {
     constexpr int kSlabs = D / 64;
     constexpr int kTileBytes = kSlabs * kSlabBytes;            // one K or V tile, also one Q half
-    constexpr int kQBytes = 2 * kTileBytes;                    // both halves of a row block
-    constexpr int kNV = (QBUF == 2) ? 1 : 2;                   // V stages
+    constexpr int kQBytes = (ALT ? 1 : 2) * kTileBytes;        // both halves of a row block (ALT: the one half both read)
+    constexpr int kNK = ALT ? 3 : 2;                           // K stages
+    constexpr int kNV = ALT ? 3 : (QBUF == 2) ? 1 : 2;         // V stages
+    static_assert(!(ALT && QBUF != 1), "alternating halves go with one Q buffer");
     constexpr uint32_t kTmemCols = 512;
     constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 256 + D;
     constexpr uint32_t kIdescQK = idesc_bf16_f32(128, kTileN, 0, 0);
@@ -121,7 +126,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int b = 0; b < QBUF; ++b) { mbar_init(bar_q_full + 8 * b, 1); mbar_init(bar_q_empty + 8 * b, 2); }   // released by both MMA issuers
-        for (int s = 0; s < kNK; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 2); }
+        for (int s = 0; s < kNK; ++s) { mbar_init(bar_k_full + 8 * s, 1); mbar_init(bar_k_empty + 8 * s, 2); }   // released by both issuers
         for (int s = 0; s < kNV; ++s) { mbar_init(bar_v_full + 8 * s, 1); mbar_init(bar_v_empty + 8 * s, 2); }
         for (int w = 0; w < 2; ++w) {
             mbar_init(bar_s_full + 8 * w, 1);
@@ -146,7 +151,8 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int group = blockIdx.x / n_sib, sib = blockIdx.x - group * n_sib;
     const int item_begin = p.cta_item_begin[group], item_end = p.cta_item_begin[group + 1];
     const int G = p.G;
-    const int TB = kAttnRows / G;            // query tokens per row block
+    constexpr bool alt = ALT;                // both halves read the same 128 rows and take alternate tiles
+    const int TB = (alt ? kHalfRows : kAttnRows) / G;            // query tokens per row block
 
     auto geom = [&](const DevItem& item, const DevReq& rq) {
         ItemGeom g;
@@ -170,7 +176,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (q_use > 0 && !mbar_wait(bar_q_empty + 8 * qb, (q_use - 1) & 1, &abort_flag, p.status)) return false;
         mbar_expect_tx(bar_q_full + 8 * qb, kQBytes);
         #pragma unroll
-        for (int w = 0; w < 2; ++w) {
+        for (int w = 0; w < (ALT ? 1 : 2); ++w) {
             const int tok0 = rq.q_row0 + g.rb * TB + w * (kHalfRows / G);
             #pragma unroll
             for (int sl = 0; sl < kSlabs; ++sl)
@@ -279,7 +285,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // Descriptors differ from their tile's base descriptor only in the 14-bit start-address field (units of 16 B),
         // so every MMA costs one add per operand instead of a descriptor build: the issuing lane shares its scheduler
         // with two softmax warps and must stay lean.
-        uint64_t q_desc0 = smem_desc_sw128(smem_u32(q_smem + w * kTileBytes), 16, 1024);
+        uint64_t q_desc0 = smem_desc_sw128(smem_u32(q_smem + (ALT ? 0 : w) * kTileBytes), 16, 1024);
         auto issue_qk = [&](uint32_t k_base) {
             const uint64_t k_desc0 = smem_desc_sw128(k_base, 16, 1024);
             #pragma unroll
@@ -366,7 +372,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 const uint32_t qb = q_loads % QBUF;
                 if (!wait_all(bar_q_full + 8 * qb, (q_loads / QBUF) & 1)) { ok = false; break; }
-                if (QBUF > 1) q_desc0 = smem_desc_sw128(smem_u32(q_smem + qb * kQBytes + w * kTileBytes), 16, 1024);
+                if (QBUF > 1) q_desc0 = smem_desc_sw128(smem_u32(q_smem + qb * kQBytes + (ALT ? 0 : w) * kTileBytes), 16, 1024);
                 ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
             }
             bool have_prev = false, o_started = false;
@@ -378,11 +384,21 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (t + 1 < item.tile_end) next_tile = p.tiles[t + 1];
                 if (!tile_visible(tile, g)) continue;
                 const int ksn = kcnt % kNK;
-                if (!wait_all(bar_k_full + 8 * ksn, (kcnt / kNK) & 1)) { ok = false; break; }
-                const uint32_t k_base = smem_u32(k_smem + ksn * kTileBytes);
-                ++kcnt;
+                const uint32_t kphase = (kcnt / kNK) & 1;
                 const uint32_t vs = vcnt % kNV, vphase = (vcnt / kNV) & 1;
-                ++vcnt;
+                const uint32_t tile_no = kcnt;                     // visible tiles of the CTA before this one
+                ++kcnt; ++vcnt;
+                if (alt && (tile_no & 1u) != static_cast<uint32_t>(w)) {
+                    // the other half's tile: this half only lets go of the stages, once they have been filled (an arrival
+                    // before that could be counted for the stage's previous tile)
+                    if (!wait_all(bar_k_full + 8 * ksn, kphase)) { ok = false; break; }
+                    if (lane == 0) mbar_arrive(bar_k_empty + 8 * ksn);
+                    if (!wait_all(bar_v_full + 8 * vs, vphase)) { ok = false; break; }
+                    if (lane == 0) mbar_arrive(bar_v_empty + 8 * vs);
+                    continue;
+                }
+                if (!wait_all(bar_k_full + 8 * ksn, kphase)) { ok = false; break; }
+                const uint32_t k_base = smem_u32(k_smem + ksn * kTileBytes);
                 if (have_prev) {
                     if (!pv_prev(prev_vs, prev_vphase, prev_valid, prev_n16, o_started)) { ok = false; break; }
                     o_started = true;
@@ -425,7 +441,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t tS = tmem_base + lane_base + (w ? kColS1 : kColS0);
         const uint32_t tO = tmem_base + lane_base + (w ? kColO1 : kColO0);
         const uint32_t my_s_full = bar_s_full + 8 * w, my_p_full = bar_p_full + 32 * w, my_o_full = bar_o_full + 8 * w;
-        uint32_t scnt = 0, ocnt = 0, q_loads = 0;
+        uint32_t scnt = 0, ocnt = 0, q_loads = 0, tcnt = 0;         // tcnt: visible tiles of the CTA so far (either half's)
         int last_req = -1, last_head = -1, last_rb = -1;
         bool ok = true;
 
@@ -438,8 +454,9 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (!(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
                 ++q_loads; last_req = item.req; last_head = item.kv_head; last_rb = g.rb;
             }
-            const int tok = g.rb * TB + R / G;
-            const int hg = R % G;
+            const int Rq = alt ? r_local : R;                       // row of the block whose query this thread holds
+            const int tok = g.rb * TB + Rq / G;
+            const int hg = Rq % G;
             const bool live = tok < rq.q_len;
             const float scale = (item.seg == SEG_CTX) ? p.scale_ctx_log2 : p.scale_oth_log2;
             float m = -INFINITY, l = 0.f;
@@ -450,6 +467,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const DevTile tile = next_tile;
                 if (t + 1 < item.tile_end) next_tile = p.tiles[t + 1];      // in flight while this tile is processed
                 if (!tile_visible(tile, g)) continue;
+                if (alt && (tcnt++ & 1u) != static_cast<uint32_t>(w)) continue;   // the other half's tile
                 if (!__all_sync(0xffffffffu, mbar_wait(my_s_full, scnt & 1, &abort_flag, p.status))) { ok = false; break; }
                 ++scnt;
                 tc_fence_after();
@@ -505,7 +523,8 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 // The two halves take turns in the exponential phase: the special-function unit is the scarcest pipe, and
                 // alternating keeps one half in its exponentials while the other half's MMAs run.  Phase n of half 0 follows
                 // phase n-1 of half 1; phase n of half 1 follows phase n of half 0 (both halves see the same tiles).
-                {
+                // (Alternating halves work on different tiles, with different numbers of them: no turns there.)
+                if (!alt) {
                     const uint32_t n = scnt - 1;
                     bool turn = true;
                     if (w == 0) { if (n > 0) turn = mbar_wait(bar_tok, (n - 1) & 1, &abort_flag, p.status); }
@@ -529,7 +548,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         sum2[i & 1] = add2(sum2[i & 1], pack2(p0, p1));
                         pk[i] = pack_bf16x2(p0, p1);
                     }
-                    if (qq == 3) {                                         // exponentials issued: the other half's turn
+                    if (qq == 3 && !alt) {                                 // exponentials issued: the other half's turn
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar_tok + 8 * (1 - w));
                     }
@@ -697,10 +716,11 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
 }
 
-size_t attn_smem_bytes(int D, int q_bufs) {
+size_t attn_smem_bytes(int D, int q_bufs, int alt) {
     const size_t tile = static_cast<size_t>(D / 64) * kSlabBytes;
-    const int tiles = (q_bufs == 2) ? (4 + kNK + 1) : (2 + kNK + 2);     // Q halves + K stages + V stages
-    return 1024 + tiles * tile + 256;
+    // Q halves + K stages + V stages
+    const int tiles = alt ? (1 + 3 + 3) : (q_bufs == 2) ? (4 + 2 + 1) : (2 + 2 + 2);
+    return 1024 + tiles * tile + 512;
 }
 
 // The register hand-over only works if the registers that the third warpgroup gives up cover what the two softmax
@@ -716,27 +736,30 @@ static cudaError_t check_register_handover(K kernel) {
     return (attr.numRegs >= kRegsOther && attr.numRegs <= kRegsSoftmax && freed >= wanted) ? cudaSuccess : cudaErrorLaunchOutOfResources;
 }
 
-cudaError_t attn_set_smem_attr(int D, int q_bufs, size_t smem_bytes) {
+template <typename K>
+static cudaError_t prepare_kernel(K kernel, int smem_bytes) {
+    const cudaError_t e = check_register_handover(kernel);
+    return e != cudaSuccess ? e : cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+}
+
+cudaError_t attn_set_smem_attr(int D, int q_bufs, int alt, size_t smem_bytes) {
     const int n = static_cast<int>(smem_bytes);
-    cudaError_t e;
-    if (D == 128 && q_bufs == 2) e = check_register_handover(ape_attn_kernel<128, 2>);
-    else if (D == 128) e = check_register_handover(ape_attn_kernel<128, 1>);
-    else if (q_bufs == 2) e = check_register_handover(ape_attn_kernel<64, 2>);
-    else e = check_register_handover(ape_attn_kernel<64, 1>);
-    if (e != cudaSuccess) return e;
-    if (D == 128 && q_bufs == 2) return cudaFuncSetAttribute(ape_attn_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
-    if (D == 128) return cudaFuncSetAttribute(ape_attn_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
-    if (q_bufs == 2) return cudaFuncSetAttribute(ape_attn_kernel<64, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
-    return cudaFuncSetAttribute(ape_attn_kernel<64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+    if (alt) return D == 128 ? prepare_kernel(ape_attn_kernel<128, 1, true>, n) : prepare_kernel(ape_attn_kernel<64, 1, true>, n);
+    if (D == 128) return q_bufs == 2 ? prepare_kernel(ape_attn_kernel<128, 2, false>, n) : prepare_kernel(ape_attn_kernel<128, 1, false>, n);
+    return q_bufs == 2 ? prepare_kernel(ape_attn_kernel<64, 2, false>, n) : prepare_kernel(ape_attn_kernel<64, 1, false>, n);
 }
 
 cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const CUtensorMap& tm_o,
                         const SplitMaps& split, const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream)
 {
-    if (D == 128 && p.n_q_bufs == 2) ape_attn_kernel<128, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
-    else if (D == 128) ape_attn_kernel<128, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
-    else if (p.n_q_bufs == 2) ape_attn_kernel<64, 2><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
-    else ape_attn_kernel<64, 1><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
+    if (p.alt_halves) {
+        if (D == 128) ape_attn_kernel<128, 1, true><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
+        else ape_attn_kernel<64, 1, true><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
+    }
+    else if (D == 128 && p.n_q_bufs == 2) ape_attn_kernel<128, 2, false><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
+    else if (D == 128) ape_attn_kernel<128, 1, false><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
+    else if (p.n_q_bufs == 2) ape_attn_kernel<64, 2, false><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
+    else ape_attn_kernel<64, 1, false><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
     return cudaGetLastError();
 }
 

@@ -51,11 +51,13 @@ struct AttnParams {
     int32_t split_r;                 // rows of a TILE_SPLIT tile that come from the prefix (a multiple of 8; 0: no such tiles)
     int32_t o_via_tma;               // two-buffer plans whose items all have their own Q: full halves of O leave through shared
                                      // memory (the item's Q buffer) and a bulk tensor store described by tm_o
+    int32_t alt_halves;              // one-buffer plans whose row blocks have 128 rows: both halves read the same rows and take
+                                     // alternate tiles; a slot then holds two partials of 128 rows (half 0, half 1)
     int* status;
 };
 
-size_t attn_smem_bytes(int D, int q_bufs);
-cudaError_t attn_set_smem_attr(int D, int q_bufs, size_t smem_bytes);
+size_t attn_smem_bytes(int D, int q_bufs, int alt);
+cudaError_t attn_set_smem_attr(int D, int q_bufs, int alt, size_t smem_bytes);
 // K and V boxes of split_r rows (prefix part) and 128 - split_r rows (context part) for TILE_SPLIT tiles
 struct SplitMaps { CUtensorMap ka, kb, va, vb; };
 cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const CUtensorMap& tm_o,

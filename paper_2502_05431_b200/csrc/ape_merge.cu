@@ -22,20 +22,39 @@ __device__ __forceinline__ void combine_segment(const float* __restrict__ ws_o, 
     M = -INFINITY; L = 0.f;
     #pragma unroll
     for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
-    for (int i = 0; i < n; ++i) {
-        const size_t slot = static_cast<size_t>(slot0) + static_cast<size_t>(i) * stride;
-        const float2 ml = *reinterpret_cast<const float2*>(ws_ml + (slot * rows_per_slot + row) * 2);
-        if (!(ml.y > 0.f)) continue;                 // empty partial
-        const float Mn = fmaxf(M, ml.x);
-        const float f_old = fast_exp2(M - Mn), f_new = fast_exp2(ml.x - Mn);
-        const float* src = ws_o + (slot * rows_per_slot + row) * D + lane * VEC;
-        float x[VEC];
-        if constexpr (VEC == 4) { const float4 t = *reinterpret_cast<const float4*>(src); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
-        else { const float2 t = *reinterpret_cast<const float2*>(src); x[0] = t.x; x[1] = t.y; }
+    // The partials are independent of each other: their loads are issued eight at a time, then folded in order (a merge
+    // with many partials per row, such as a decode batch that shares its contexts, is bound by the latency of these loads).
+    constexpr int kBatch = 8;
+    for (int i0 = 0; i0 < n; i0 += kBatch) {
+        float2 ml[kBatch];
+        float x[kBatch][VEC];
         #pragma unroll
-        for (int v = 0; v < VEC; ++v) acc[v] = acc[v] * f_old + x[v] * f_new;
-        L = L * f_old + ml.y * f_new;
-        M = Mn;
+        for (int u = 0; u < kBatch; ++u) {
+            const size_t slot = static_cast<size_t>(slot0) + static_cast<size_t>(i0 + u) * stride;
+            ml[u] = (i0 + u < n) ? *reinterpret_cast<const float2*>(ws_ml + (slot * rows_per_slot + row) * 2) : make_float2(-INFINITY, 0.f);
+        }
+        #pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const size_t slot = static_cast<size_t>(slot0) + static_cast<size_t>(i0 + u) * stride;
+            const float* src = ws_o + (slot * rows_per_slot + row) * D + lane * VEC;
+            if (ml[u].y > 0.f) {                     // an empty partial's rows were never written
+                if constexpr (VEC == 4) { const float4 t = *reinterpret_cast<const float4*>(src); x[u][0] = t.x; x[u][1] = t.y; x[u][2] = t.z; x[u][3] = t.w; }
+                else { const float2 t = *reinterpret_cast<const float2*>(src); x[u][0] = t.x; x[u][1] = t.y; }
+            } else {
+                #pragma unroll
+                for (int v = 0; v < VEC; ++v) x[u][v] = 0.f;
+            }
+        }
+        #pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            if (!(ml[u].y > 0.f)) continue;          // empty partial
+            const float Mn = fmaxf(M, ml[u].x);
+            const float f_old = fast_exp2(M - Mn), f_new = fast_exp2(ml[u].x - Mn);
+            #pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[v] = acc[v] * f_old + x[u][v] * f_new;
+            L = L * f_old + ml[u].y * f_new;
+            M = Mn;
+        }
     }
 }
 

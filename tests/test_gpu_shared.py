@@ -29,6 +29,9 @@ def _check(b, kv_extra=0, lse_tol=2e-3):
     (dict(H_q=16, H_kv=1, d=128, l_P=64, ctx_lens=[256] * 3, l_k=65, T=1.1, S=0.9), 20),    # G = 16: two row blocks
     (dict(**LLAMA, l_P=4, ctx_lens=[], l_k=3, T=0.9, S=0.9), 2),                            # no contexts at all
     (dict(**LLAMA, l_P=0, ctx_lens=[129], l_k=1, T=0.8, S=0.7), 70),                        # 70 x 4 rows: two row blocks, ragged
+    (dict(**LLAMA, l_P=5, ctx_lens=[100], l_k=2, T=0.9, S=0.9), 32),                        # 128 rows exactly, one tile: one half idle
+    (dict(**LLAMA, l_P=5, ctx_lens=[100, 700], l_k=2, T=0.9, S=0.9), 33),                   # 132 rows: one 256-row block again
+    (dict(**LLAMA, l_P=9, ctx_lens=[128 * 5], l_k=2, T=0.7, S=0.8), 9),                     # an odd number of whole tiles
 ])
 def test_shared_context_decode(kw, n_req):
     lens = kw.pop("ctx_lens")
