@@ -715,8 +715,12 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
     p->split_r = split_r;
     HostMeta m;
     try {
+        // The row blocks of one (context, KV head) read the same K/V tiles: a pair's row blocks go to ONE CTA, back to back
+        // (the longest, which touches every tile of the context, first), so the tiles come from HBM once and from L2 for the
+        // other row blocks.  Whole pairs are dealt out while every CTA gets the same number; the rest goes item by item.
         struct Work { DevItem it; long long cost; };
-        std::vector<Work> work;
+        struct Pair { std::vector<Work> rows; long long cost; };
+        std::vector<Pair> pairs;
         for (int i = 0; i < n_ctx; ++i) {
             DevReq dr{static_cast<int32_t>(ctx[i].start), static_cast<int32_t>(ctx[i].len), static_cast<int32_t>(ctx[i].len), 0};
             m.reqs.push_back(dr);
@@ -747,8 +751,9 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
             }
             const int t1 = static_cast<int>(m.tiles.size());
             const int RB = static_cast<int>((ctx[i].len + TB - 1) / TB);
-            for (int hh = 0; hh < H_kv; ++hh)
-                for (int rb = 0; rb < RB; ++rb) {
+            for (int hh = 0; hh < H_kv; ++hh) {
+                Pair pr; pr.cost = 0;
+                for (int rb = RB - 1; rb >= 0; --rb) {
                     const int64_t last_tok = std::min<int64_t>(ctx[i].len, static_cast<int64_t>(rb + 1) * TB) - 1;
                     // tiles this row block can see: the prefix tiles and every context tile whose first key is not past last_tok
                     const int vis = (split_r > 0)
@@ -757,18 +762,28 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
                     DevItem it{};
                     it.req = i; it.kv_head = hh; it.row_block = rb; it.tile_begin = t0; it.tile_end = std::min(t1, t0 + vis);
                     it.slot = 0; it.seg = SEG_FINAL; it.n_sib = 1;
-                    work.push_back(Work{it, vis});
+                    pr.rows.push_back(Work{it, vis}); pr.cost += vis;
                 }
+                pairs.push_back(std::move(pr));
+            }
         }
-        // longest-first round robin over the CTAs keeps the per-CTA tile counts close
-        std::stable_sort(work.begin(), work.end(), [](const Work& a, const Work& b) { return a.cost > b.cost; });
-        p->n_cta = std::max(1, std::min<int>(h->n_sm, static_cast<int>(work.size())));
+        size_t n_items = 0;
+        for (auto& pr : pairs) n_items += pr.rows.size();
+        p->n_cta = std::max(1, std::min<int>(h->n_sm, static_cast<int>(n_items)));
         std::vector<std::vector<DevItem>> bins(p->n_cta);
         std::vector<long long> load(p->n_cta, 0);
-        for (size_t w = 0; w < work.size(); ++w) {
-            int b = static_cast<int>(std::min_element(load.begin(), load.end()) - load.begin());
-            bins[b].push_back(work[w].it); load[b] += work[w].cost;
+        auto least = [&]() { return static_cast<int>(std::min_element(load.begin(), load.end()) - load.begin()); };
+        std::stable_sort(pairs.begin(), pairs.end(), [](const Pair& a, const Pair& b) { return a.cost > b.cost; });
+        const size_t whole = pairs.size() / p->n_cta * p->n_cta;      // pairs dealt out whole, longest first
+        for (size_t i = 0; i < whole; ++i) {
+            const int b = least();
+            for (auto& w : pairs[i].rows) bins[b].push_back(w.it);
+            load[b] += pairs[i].cost;
         }
+        std::vector<Work> rest;
+        for (size_t i = whole; i < pairs.size(); ++i) for (auto& w : pairs[i].rows) rest.push_back(w);
+        std::stable_sort(rest.begin(), rest.end(), [](const Work& a, const Work& b) { return a.cost > b.cost; });
+        for (auto& w : rest) { const int b = least(); bins[b].push_back(w.it); load[b] += w.cost; }
         m.cta_begin.push_back(0);
         for (auto& b : bins) { for (auto& it : b) m.items.push_back(it); m.cta_begin.push_back(static_cast<int32_t>(m.items.size())); }
         p->n_slots = 0;
