@@ -588,6 +588,15 @@ def main():
 
     pre, enc = tensor_leg(t["prefill"], fl_prefill), tensor_leg(t["encode"], fl_encode)
     pre["ms_mean"], enc["ms_mean"] = t_mean["prefill"], t_mean["encode"]
+    # Encode of short contexts moves Q in and O out once per row and K/V once per context: by the roofline of the measured
+    # peaks it is bound by HBM, not by the tensor cores, whenever its FLOP per algorithmic byte sit below the ridge.
+    enc_bytes = 2 * 2.0 * N_CTX * L_CTX * H_Q * D + (L_P + N_CTX * L_CTX) * 4.0 * H_KV * D
+    enc_gbs = enc_bytes / (t["encode"] * 1e-3) / 1e9
+    ridge = peaks["tf_burst"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    enc["roofline"] = {"bound": "hbm" if fl_encode / enc_bytes < ridge else "tensor", "algorithmic_bytes": enc_bytes,
+                       "flop_per_byte": fl_encode / enc_bytes, "ridge_flop_per_byte": ridge, "achieved": enc_gbs, "peak": peaks["hbm_gbs"],
+                       "unit": "GB/s", "frac": enc_gbs / peaks["hbm_gbs"], "traffic": None,
+                       "what": "Q read + O written once per row, K/V read once per context; the tensor fractions above are the other bound"}
     tf_prefill = pre["tflops"]
     gbs_decode = by_decode_total / (dec_total_ms * 1e-3) / 1e9
     roof = {"bound": "tensor", "kernel": "ape_attn_kernel<128,1> (+ merge) on the 128K prefill", "achieved": tf_prefill,
