@@ -59,7 +59,14 @@ struct ape_plan_s {
     bool alt_halves = false;        // context pass of a shared plan with at most 128 rows: the halves take alternate tiles
     int32_t last_launches = 0;
     int per_context = 0;             // merge form: 0 Eq. 5, 1 Eq. 11-12 (per context), 2 context trees
-    DevNode* d_nodes = nullptr;      // tree plans
+    DevNode* d_nodes = nullptr;      // tree plans; two-pass plans
+    // Prefill plans of the per-context and tree forms run in two passes (statistics of every node's own tokens, then
+    // the prefill with per-row, per-node biases): their per-node arrays live behind the partials in the workspace.
+    bool two_pass = false;
+    int32_t* d_req_node0 = nullptr;  // [n_req + 1]
+    int n_nodes = 0, max_rows = 0, max_nodes = 0;
+    int64_t stat_rows = 0;
+    size_t off_stats = 0, off_mass = 0, off_bias = 0;
     // shared-context decode plans: the context pass of all requests (tensor-core kernel) and the per-request rest (decode kernel)
     ape_plan_s* child_ctx = nullptr;
     ape_plan_s* child_oth = nullptr;
@@ -205,7 +212,8 @@ struct HostMeta {
     std::vector<int32_t> cta_begin;
     std::vector<DevReq> reqs;
     std::vector<DevMerge> merge;
-    std::vector<DevNode> nodes;      // tree plans
+    std::vector<DevNode> nodes;      // tree plans; two-pass plans
+    std::vector<int32_t> req_node0;  // two-pass plans: first node of every request, and the total
 };
 
 struct Run {   // a run of tiles of one segment for one (request, kv head, row-block group)
@@ -215,7 +223,9 @@ struct Run {   // a run of tiles of one segment for one (request, kv head, row-b
 
 // Split the concatenation of all runs evenly over n_bins bins (each bin = one CTA or one sibling group);
 // a run that straddles a bin boundary becomes several items, each with its own partial slot.
-void assign_stream(const std::vector<Run>& runs, int n_bins, int slot_mult, HostMeta& m) {
+// With align_nodes (two-pass plans) a context run is only cut behind a tile that ends a node: the statistics pass keeps a
+// node's running (maximum, sum) in registers and writes it once, so a node's tiles must not be spread over two items.
+void assign_stream(const std::vector<Run>& runs, int n_bins, int slot_mult, HostMeta& m, bool align_nodes = false) {
     long long total = 0;
     for (const auto& r : runs) total += r.t1 - r.t0;
     const long long chunk = std::max<long long>(1, (total + n_bins - 1) / n_bins);
@@ -224,7 +234,9 @@ void assign_stream(const std::vector<Run>& runs, int n_bins, int slot_mult, Host
     for (const auto& r : runs) {
         int t = r.t0;
         while (t < r.t1) {
-            const int take = static_cast<int>(std::min<long long>(room, r.t1 - t));
+            int take = static_cast<int>(std::min<long long>(room, r.t1 - t));
+            if (align_nodes && r.seg == SEG_CTX)
+                while (t + take < r.t1 && !(m.tiles[t + take - 1].flags & TILE_CTX_END)) ++take;
             DevItem it;
             it.req = r.req; it.kv_head = r.kv_head; it.row_block = r.row_block;
             it.tile_begin = t; it.tile_end = t + take;
@@ -239,7 +251,7 @@ void assign_stream(const std::vector<Run>& runs, int n_bins, int slot_mult, Host
             }
             m.items.push_back(it);
             t += take; room -= take;
-            if (room == 0) { m.cta_begin.push_back(static_cast<int32_t>(m.items.size())); room = chunk; }
+            if (room <= 0) { m.cta_begin.push_back(static_cast<int32_t>(m.items.size())); room = chunk; }
         }
     }
     while (static_cast<int>(m.cta_begin.size()) < n_bins + 1) m.cta_begin.push_back(static_cast<int32_t>(m.items.size()));
@@ -259,8 +271,9 @@ int upload(ape_plan_t p, const HostMeta& m) {
     auto rnd = [](size_t x) { return (x + 255) & ~size_t(255); };
     const size_t b_tiles = rnd(m.tiles.size() * sizeof(DevTile) + 16), b_items = rnd(m.items.size() * sizeof(DevItem) + 16),
                  b_cta = rnd(m.cta_begin.size() * 4 + 16), b_reqs = rnd(m.reqs.size() * sizeof(DevReq) + 16),
-                 b_merge = rnd(m.merge.size() * sizeof(DevMerge) + 16), b_nodes = rnd(m.nodes.size() * sizeof(DevNode) + 16);
-    const size_t total = b_tiles + b_items + b_cta + b_reqs + b_merge + b_nodes;
+                 b_merge = rnd(m.merge.size() * sizeof(DevMerge) + 16), b_nodes = rnd(m.nodes.size() * sizeof(DevNode) + 16),
+                 b_rn = rnd(m.req_node0.size() * 4 + 16);
+    const size_t total = b_tiles + b_items + b_cta + b_reqs + b_merge + b_nodes + b_rn;
     std::vector<uint8_t> host(total, 0);
     size_t o = 0;
     auto put = [&](const void* src, size_t n, size_t padded) { if (n) std::memcpy(host.data() + o, src, n); size_t at = o; o += padded; return at; };
@@ -270,6 +283,7 @@ int upload(ape_plan_t p, const HostMeta& m) {
     const size_t o_reqs = put(m.reqs.data(), m.reqs.size() * sizeof(DevReq), b_reqs);
     const size_t o_merge = put(m.merge.data(), m.merge.size() * sizeof(DevMerge), b_merge);
     const size_t o_nodes = put(m.nodes.data(), m.nodes.size() * sizeof(DevNode), b_nodes);
+    const size_t o_rn = put(m.req_node0.data(), m.req_node0.size() * 4, b_rn);
     if (cudaMalloc(&p->d_blob, total) != cudaSuccess) { p->d_blob = nullptr; return APE_ERR_NOMEM; }
     if (cudaMemcpy(p->d_blob, host.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) return APE_ERR_CUDA;
     uint8_t* b = static_cast<uint8_t*>(p->d_blob);
@@ -279,6 +293,7 @@ int upload(ape_plan_t p, const HostMeta& m) {
     p->d_reqs = reinterpret_cast<DevReq*>(b + o_reqs);
     p->d_merge = reinterpret_cast<DevMerge*>(b + o_merge);
     p->d_nodes = reinterpret_cast<DevNode*>(b + o_nodes);
+    p->d_req_node0 = reinterpret_cast<int32_t*>(b + o_rn);
     p->n_items = static_cast<int>(m.items.size());
     p->n_merge = static_cast<int>(m.merge.size());
     return APE_OK;
@@ -418,6 +433,17 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
             return APE_ERR_NOMEM;
         }
     }
+    if (per_context == 1 && mode != APE_DECODE) {
+        // Eq. 11-12 as a forest of depth 0: every context a marked top-level node (the prefill plan runs in two passes)
+        try {
+            for (int r = 0; r < n_req; ++r) {
+                node_base[r] = static_cast<int>(m.nodes.size());
+                for (int i = 0; i < reqs[r].n_ctx; ++i) m.nodes.push_back(DevNode{-1, 0, 1, 0});
+            }
+        } catch (const std::bad_alloc&) {
+            return APE_ERR_NOMEM;
+        }
+    }
     DeviceGuard guard(h->device);
     if (!guard.ok) return APE_ERR_CUDA;
 
@@ -426,6 +452,7 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
     p->h = h; p->kind = (mode == APE_DECODE) ? PLAN_DECODE : PLAN_PREFILL;
     p->shape = *shape; p->c = c; p->G = G; p->pool = *pool; p->q = *q; p->out = *out; p->lse = lse; p->per_context = per_context;
     p->max_kv_extra = (mode == APE_DECODE) ? max_extra : 0;
+    p->n_req = n_req;
     const int D = shape->head_dim, H_kv = shape->n_kv_heads;
 
     std::vector<Run> runs;
@@ -472,16 +499,44 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
             for (int r = 0; r < n_req; ++r) max_rb = std::max<int>(max_rb, static_cast<int>((reqs[r].q_len + TB - 1) / TB));
             p->n_sib = std::max(1, std::min({4, max_rb, h->n_sm}));
             const int n_groups = std::max(1, h->n_sm / p->n_sib);
+            int64_t row_base = 0;                          // query rows of the requests before this one
+            bool any_node_tiles = false;
             for (int r = 0; r < n_req; ++r) {
                 const ape_request_t& rq = reqs[r];
-                DevReq dr{static_cast<int32_t>(rq.q_start), static_cast<int32_t>(rq.q_len), static_cast<int32_t>(rq.query_kv.len), 0};
+                // (pad: the request's row base, which the two-pass plans index their per-node arrays with)
+                DevReq dr{static_cast<int32_t>(rq.q_start), static_cast<int32_t>(rq.q_len), static_cast<int32_t>(rq.query_kv.len),
+                          static_cast<int32_t>(row_base)};
                 m.reqs.push_back(dr);
+                m.req_node0.push_back(node_base[r]);
+                p->max_nodes = std::max(p->max_nodes, rq.n_ctx);
                 const int o0 = static_cast<int>(m.tiles.size());
                 add_span_tiles(m.tiles, rq.prefix.start, rq.prefix.len, tile, 0, 0);
                 add_span_tiles(m.tiles, rq.query_kv.start, rq.query_kv.len, tile, TILE_CAUSAL, 0);
                 const int o1 = static_cast<int>(m.tiles.size());
-                const auto ctx_ranges = (per_context == 2) ? add_tree_tiles(m.tiles, rq.ctx, parent[r], rq.n_ctx, tile, node_base[r])
-                                                            : add_context_tiles(m.tiles, rq.ctx, rq.n_ctx, tile, per_context == 1);
+                std::vector<CtxRange> ctx_ranges;
+                if (per_context == 2) ctx_ranges = add_tree_tiles(m.tiles, rq.ctx, parent[r], rq.n_ctx, tile, node_base[r]);
+                else if (per_context == 1) {
+                    for (int i = 0; i < rq.n_ctx; ++i) {
+                        if (rq.ctx[i].len <= 0) continue;
+                        const int c0 = static_cast<int>(m.tiles.size());
+                        add_span_tiles(m.tiles, rq.ctx[i].start, rq.ctx[i].len, tile, 0, 0);
+                        ctx_ranges.push_back({c0, static_cast<int>(m.tiles.size()), node_base[r] + i});
+                    }
+                } else ctx_ranges = add_context_tiles(m.tiles, rq.ctx, rq.n_ctx, tile, false);
+                if (per_context != 0 && !ctx_ranges.empty()) {
+                    // Two passes instead of a partial per node: every context tile names its node (key_base is free, these
+                    // tiles are not causal) and a node's last tile is marked; the context segment is then ONE run of tiles
+                    // (the ranges follow each other in the tile list), as in the Eq. 5 plan, and long items stay long.
+                    for (const auto& cr : ctx_ranges) {
+                        for (int t = cr.t0; t < cr.t1; ++t) m.tiles[t].key_base = cr.id;
+                        m.tiles[cr.t1 - 1].flags |= TILE_CTX_END;
+                        m.nodes[cr.id].pad = 1;
+                    }
+                    ctx_ranges = {CtxRange{ctx_ranges.front().t0, ctx_ranges.back().t1, static_cast<int>(row_base)}};
+                    any_node_tiles = true;
+                }
+                row_base += rq.q_len;
+                p->max_rows = std::max<int>(p->max_rows, static_cast<int>(rq.q_len) * shape->n_q_heads);
                 const int RB = static_cast<int>((rq.q_len + TB - 1) / TB);
                 for (int hh = 0; hh < H_kv; ++hh) {
                     for (int rb0 = 0; rb0 < RB; rb0 += p->n_sib) {
@@ -494,16 +549,31 @@ static int attend_plan_impl(ape_handle_t h, const ape_shape_t* shape, const ape_
                     }
                 }
             }
-            assign_stream(runs, n_groups, p->n_sib, m);
+            assign_stream(runs, n_groups, p->n_sib, m, per_context != 0);
             p->n_cta = n_groups * p->n_sib;
             p->n_slots = static_cast<int>(m.items.size()) * p->n_sib;
-            p->smem_bytes = attn_smem_bytes(D, 1, 0);
+            p->smem_bytes = attn_smem_bytes(D, kAttnPrefill);
             const size_t rows = static_cast<size_t>(p->n_slots) * kAttnRows;
             p->ws_bytes = ((rows * D * 4 + 255) & ~size_t(255)) + ((rows * 2 * 4 + 255) & ~size_t(255));
+            m.req_node0.push_back(static_cast<int32_t>(m.nodes.size()));
+            if (per_context != 0 && any_node_tiles) {
+                if (row_base * shape->n_q_heads >= (1ll << 31)) { delete p; return APE_ERR_LAYOUT; }
+                p->two_pass = true;
+                p->n_nodes = static_cast<int>(m.nodes.size());
+                p->stat_rows = row_base * shape->n_q_heads;
+                const size_t cells = static_cast<size_t>(p->n_nodes) * static_cast<size_t>(p->stat_rows);
+                auto rnd = [](size_t x) { return (x + 255) & ~size_t(255); };
+                p->off_stats = p->ws_bytes;
+                p->off_mass = p->off_stats + rnd(cells * 8);
+                p->off_bias = p->off_mass + rnd(cells * 4);
+                p->ws_bytes = p->off_bias + rnd(cells * 4);
+            }
             rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
             if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
             if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
-            if (!rc && attn_set_smem_attr(D, 1, 0, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+            if (!rc && attn_set_smem_attr(D, kAttnPrefill, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+            if (!rc && p->two_pass && (attn_set_smem_attr(D, kAttnStats, p->smem_bytes) != cudaSuccess ||
+                                       attn_set_smem_attr(D, kAttnBias, p->smem_bytes) != cudaSuccess)) rc = APE_ERR_CUDA;
         }
         if (!rc) { finish_items(m); rc = upload(p, m); }
     } catch (const std::bad_alloc&) {
@@ -608,11 +678,11 @@ int ape_attend_plan_shared(ape_handle_t h, const ape_shape_t* shape, const ape_k
         assign_stream(runs_a, n_groups, a->n_sib, ma);
         a->n_cta = n_groups * a->n_sib;
         a->n_slots = static_cast<int>(ma.items.size()) * a->n_sib;
-        a->smem_bytes = attn_smem_bytes(D, 1, a->alt_halves ? 1 : 0);
+        a->smem_bytes = attn_smem_bytes(D, a->alt_halves ? kAttnAlt : kAttnPrefill);
         rc = make_map(h, &a->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, kAttnTileN);
         if (!rc) rc = make_map(h, &a->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, kAttnTileN);
         if (!rc) rc = make_map(h, &a->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
-        if (!rc && attn_set_smem_attr(D, 1, a->alt_halves ? 1 : 0, a->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+        if (!rc && attn_set_smem_attr(D, a->alt_halves ? kAttnAlt : kAttnPrefill, a->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
         if (!rc) { finish_items(ma); rc = upload(a, ma); }
 
         // ---- the rest, per request: prefix + the request's own (growing) query segment ------------------------------
@@ -788,7 +858,7 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
         for (auto& b : bins) { for (auto& it : b) m.items.push_back(it); m.cta_begin.push_back(static_cast<int32_t>(m.items.size())); }
         p->n_slots = 0;
         p->ws_bytes = 0;
-        p->smem_bytes = attn_smem_bytes(D, 2, 0);
+        p->smem_bytes = attn_smem_bytes(D, kAttnEncode);
         rc = make_map(h, &p->tm_k, pool->k, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
         if (!rc) rc = make_map(h, &p->tm_v, pool->v, D, H_kv, pool->n_tokens, pool->head_stride, pool->token_stride, 1, tile);
         if (!rc) rc = make_map(h, &p->tm_q, q->data, D, shape->n_q_heads, q->n_rows, q->head_stride, q->token_stride, G, 128 / G);
@@ -801,7 +871,7 @@ int ape_encode_plan(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_
         // Every item of this plan has a row block of its own, so a finished row block may leave through its Q buffer.
         if (!rc) p->o_via_tma = make_map(h, &p->tm_o, out->data, D, shape->n_q_heads, out->n_rows, out->head_stride, out->token_stride,
                                          G, 128 / G) == APE_OK;
-        if (!rc && attn_set_smem_attr(D, 2, 0, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
+        if (!rc && attn_set_smem_attr(D, kAttnEncode, p->smem_bytes) != cudaSuccess) rc = APE_ERR_CUDA;
         if (!rc) { finish_items(m); rc = upload(p, m); }
     } catch (const std::bad_alloc&) {
         rc = APE_ERR_NOMEM;
@@ -938,8 +1008,8 @@ static int attend_impl(ape_plan_t p, float T, float S, int64_t kv_extra, void* w
             ap.tiles = a->d_tiles; ap.items = a->d_items; ap.cta_item_begin = a->d_cta_begin; ap.reqs = a->d_reqs;
             ap.out = rows_desc(p->out); ap.lse_out = nullptr; ap.ws_o = a_o; ap.ws_ml = a_ml;
             ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c / T * kLog2e;
-            ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = a->n_sib; ap.n_q_bufs = 1; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
-            ap.o_via_tma = 0; ap.split_r = 0; ap.alt_halves = a->alt_halves ? 1 : 0;
+            ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = a->n_sib; ap.mode = kAttnPrefill; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
+            ap.o_via_tma = 0; ap.split_r = 0; ap.stats = nullptr; ap.bias = nullptr; ap.stat_rows = 0; if (a->alt_halves) ap.mode = kAttnAlt;
             if (launch_attn(D, a->tm_q, a->tm_k, a->tm_v, a->tm_q, a->tm_split, ap, a->n_cta, a->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
             p->last_launches++;
         }
@@ -979,17 +1049,34 @@ static int attend_impl(ape_plan_t p, float T, float S, int64_t kv_extra, void* w
         ap.tiles = p->d_tiles; ap.items = p->d_items; ap.cta_item_begin = p->d_cta_begin; ap.reqs = p->d_reqs;
         ap.out = rows_desc(p->out); ap.lse_out = nullptr; ap.ws_o = ws_o; ap.ws_ml = ws_ml;
         ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c / T * kLog2e;
-        ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = p->n_sib; ap.n_q_bufs = 1; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
-        ap.o_via_tma = 0; ap.split_r = 0; ap.alt_halves = 0;
+        ap.G = G; ap.H_q = p->shape.n_q_heads; ap.n_sib = p->n_sib; ap.mode = kAttnPrefill; ap.q_rows_are_pool = 0; ap.status = p->h->d_status;
+        ap.o_via_tma = 0; ap.split_r = 0; ap.stats = nullptr; ap.bias = nullptr; ap.stat_rows = 0;
+        if (p->two_pass) {
+            // per-context form / context trees: (1) every node's own (maximum, sum) per row, (2) per-row, per-node biases
+            // from them and S, (3) the prefill with the biases on the context logits; the merge below then sees an
+            // ordinary context segment whose scaling has been applied already
+            uint8_t* base = static_cast<uint8_t*>(workspace);
+            ap.stat_rows = p->stat_rows;
+            ap.mode = kAttnStats; ap.stats = reinterpret_cast<float2*>(base + p->off_stats);
+            if (launch_attn(D, p->tm_q, p->tm_k, p->tm_v, p->tm_q, p->tm_split, ap, p->n_cta, p->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
+            NodeBiasParams nb;
+            nb.nodes = p->d_nodes; nb.reqs = p->d_reqs; nb.req_node0 = p->d_req_node0; nb.n_req = static_cast<int32_t>(p->n_req);
+            nb.stats = ap.stats; nb.mass = reinterpret_cast<float*>(base + p->off_mass); nb.bias = reinterpret_cast<float*>(base + p->off_bias);
+            nb.stat_rows = p->stat_rows; nb.S = S; nb.H_q = p->shape.n_q_heads; nb.max_rows = p->max_rows;
+            nb.max_nodes = p->max_nodes; nb.smem_limit = p->h->smem_optin;
+            if (launch_node_bias(nb, stream) != cudaSuccess) return APE_ERR_CUDA;
+            ap.mode = kAttnBias; ap.stats = nullptr; ap.bias = nb.bias;
+            p->last_launches += 2;
+        }
         if (launch_attn(D, p->tm_q, p->tm_k, p->tm_v, p->tm_q, p->tm_split, ap, p->n_cta, p->smem_bytes, stream) != cudaSuccess) return APE_ERR_CUDA;
     }
     p->last_launches++;
 
     MergeParams mp;
-    mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.items = p->d_items; mp.per_context = p->per_context; mp.nodes = p->d_nodes; mp.n_groups = p->n_merge; mp.rows_per_slot = rows_per_slot;
+    mp.groups = p->d_merge; mp.reqs = p->d_reqs; mp.items = p->d_items; mp.per_context = p->two_pass ? 0 : p->per_context; mp.nodes = p->d_nodes; mp.n_groups = p->n_merge; mp.rows_per_slot = rows_per_slot;
     mp.tokens_per_block = rows_per_slot / G; mp.ws_o = ws_o; mp.ws_ml = ws_ml; mp.out = rows_desc(p->out); mp.lse_out = p->lse;
     mp.ws_o_ctx = ws_o; mp.ws_ml_ctx = ws_ml; mp.rows_per_slot_ctx = rows_per_slot;
-    mp.S = S; mp.G = G; mp.H_q = p->shape.n_q_heads; mp.D = D;
+    mp.S = p->two_pass ? 1.f : S; mp.G = G; mp.H_q = p->shape.n_q_heads; mp.D = D;
     mp.part_o_ctx = part ? part->o_ctx : nullptr; mp.part_lse_ctx = part ? part->lse_ctx : nullptr;
     mp.part_o_oth = part ? part->o_oth : nullptr; mp.part_lse_oth = part ? part->lse_oth : nullptr;
     if (launch_merge(mp, stream) != cudaSuccess) return APE_ERR_CUDA;
@@ -1039,8 +1126,8 @@ int ape_encode_contexts(ape_plan_t p, void* workspace, size_t ws_bytes, void* st
     ap.tiles = p->d_tiles; ap.items = p->d_items; ap.cta_item_begin = p->d_cta_begin; ap.reqs = p->d_reqs;
     ap.out = rows_desc(p->out); ap.lse_out = p->lse; ap.ws_o = nullptr; ap.ws_ml = nullptr;
     ap.scale_oth_log2 = p->c * kLog2e; ap.scale_ctx_log2 = p->c * kLog2e;
-    ap.G = p->G; ap.H_q = p->shape.n_q_heads; ap.n_sib = 1; ap.n_q_bufs = 2; ap.q_rows_are_pool = 1; ap.status = p->h->d_status;
-    ap.o_via_tma = p->o_via_tma ? 1 : 0; ap.split_r = p->split_r; ap.alt_halves = 0;
+    ap.G = p->G; ap.H_q = p->shape.n_q_heads; ap.n_sib = 1; ap.mode = kAttnEncode; ap.q_rows_are_pool = 1; ap.status = p->h->d_status;
+    ap.o_via_tma = p->o_via_tma ? 1 : 0; ap.split_r = p->split_r; ap.stats = nullptr; ap.bias = nullptr; ap.stat_rows = 0;
     if (launch_attn(p->shape.head_dim, p->tm_q, p->tm_k, p->tm_v, p->tm_o, p->tm_split, ap, p->n_cta, p->smem_bytes,
                     static_cast<cudaStream_t>(stream_v)) != cudaSuccess) return APE_ERR_CUDA;
     p->last_launches = 1;

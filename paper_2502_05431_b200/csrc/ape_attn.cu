@@ -84,7 +84,11 @@ __device__ __forceinline__ bool tile_visible(const DevTile& t, const ItemGeom& g
 // QBUF: number of Q buffers.  Plans with long items (prefill) use one Q buffer and two stages each of K and V; plans
 // with many short items (encode) use two Q buffers, so that the next row block's Q arrives while the current one is
 // in use, and pay for them with a single V stage.
-template <int D, int QBUF, bool ALT>
+// MODE selects the configuration (ape_kernels.h): kAttnPrefill, kAttnEncode (two Q buffers), kAttnAlt (alternating halves),
+// and the two passes of the plans that scale parts of the context segment separately (per-context form, context trees):
+// kAttnStats computes, per row, the (maximum, sum) of every node's own tokens (S = Q K^T and the softmax sums only: no P,
+// no V, no O); kAttnBias is the prefill pass with a per-row, per-node bias added to the context logits.
+template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -92,10 +96,11 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 {
     constexpr int kSlabs = D / 64;
     constexpr int kTileBytes = kSlabs * kSlabBytes;            // one K or V tile, also one Q half
+    constexpr int QBUF = (MODE == kAttnEncode) ? 2 : 1;
+    constexpr bool ALT = MODE == kAttnAlt, STATS = MODE == kAttnStats, BIAS = MODE == kAttnBias;
     constexpr int kQBytes = (ALT ? 1 : 2) * kTileBytes;        // both halves of a row block (ALT: the one half both read)
     constexpr int kNK = ALT ? 3 : 2;                           // K stages
     constexpr int kNV = ALT ? 3 : (QBUF == 2) ? 1 : 2;         // V stages
-    static_assert(!(ALT && QBUF != 1), "alternating halves go with one Q buffer");
     constexpr uint32_t kTmemCols = 512;
     constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO0 = 256, kColO1 = 256 + D;
     constexpr uint32_t kIdescQK = idesc_bf16_f32(128, kTileN, 0, 0);
@@ -198,6 +203,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const DevItem item = p.items[it];
                 if (it + 1 < item_end) prefetch_l1(&p.items[it + 1]);   // the next item's record is in cache when its turn comes
                 if (sib >= item.n_sib) continue;
+                if (STATS && item.seg != SEG_CTX) continue;             // the statistics pass is about context nodes only
                 const DevReq rq{item.q_row0, item.q_len, item.l_k, 0};
                 const ItemGeom g = geom(item, rq);
                 if (QBUF == 1 && !(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
@@ -229,7 +235,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                                         sl * 64, item.kv_head, tile.tok);
                         ++kcnt;
                     }
-                    {
+                    if (!STATS) {
                         const int s = vcnt % kNV; const uint32_t use = vcnt / kNV;
                         if (!mbar_wait(bar_v_empty + 8 * s, (use & 1) ^ 1, &abort_flag, p.status)) { ok = false; break; }
                         mbar_expect_tx(bar_v_full + 8 * s, kTileBytes);
@@ -325,6 +331,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         };
         // O += P V for the previous tile of this half, in two key halves as P is published
         uint32_t prev_v_release = 0, pending_q_release = 0;
+        bool s_pending = false;                                   // statistics pass: an S tile that has not been read yet
         auto pv_prev = [&](uint32_t prev_vs, uint32_t prev_vphase, int prev_valid, int prev_n16, bool o_started) {
             if (!wait_all(bar_v_full + 8 * prev_vs, prev_vphase)) return false;
             uint8_t* v_tile = v_smem + prev_vs * kTileBytes;
@@ -359,6 +366,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const DevItem item = p.items[it];
             if (it + 1 < item_end) prefetch_l1(&p.items[it + 1]);       // the next item's record is in cache when its turn comes
             if (sib >= item.n_sib) continue;
+            if (STATS && item.seg != SEG_CTX) continue;
             const DevReq rq{item.q_row0, item.q_len, item.l_k, 0};
             const ItemGeom g = geom(item, rq);
             if (!(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
@@ -399,6 +407,20 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 if (!wait_all(bar_k_full + 8 * ksn, kphase)) { ok = false; break; }
                 const uint32_t k_base = smem_u32(k_smem + ksn * kTileBytes);
+                if (STATS) {
+                    // no product with V in this pass: the next S may be written once the softmax threads have read the
+                    // previous one into registers (they say so on the first of the P barriers), also across items
+                    if (s_pending) {
+                        if (!wait_all(my_p_full, pcnt & 1)) { ok = false; break; }
+                        ++pcnt;
+                    }
+                    tc_fence_after();
+                    issue_qk(k_base);
+                    mma_commit_elect(leader, my_s_full);
+                    mma_commit_elect(leader, bar_k_empty + 8 * ksn);
+                    s_pending = true;
+                    continue;
+                }
                 if (have_prev) {
                     if (!pv_prev(prev_vs, prev_vphase, prev_valid, prev_n16, o_started)) { ok = false; break; }
                     o_started = true;
@@ -449,6 +471,7 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const DevItem item = p.items[it];
             if (it + 1 < item_end) prefetch_l1(&p.items[it + 1]);       // the next item's record is in cache when its turn comes
             if (sib >= item.n_sib) continue;
+            if (STATS && item.seg != SEG_CTX) continue;
             const DevReq rq{item.q_row0, item.q_len, item.l_k, 0};
             const ItemGeom g = geom(item, rq);
             if (!(item.req == last_req && item.kv_head == last_head && g.rb == last_rb)) {
@@ -461,6 +484,11 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const float scale = (item.seg == SEG_CTX) ? p.scale_ctx_log2 : p.scale_oth_log2;
             float m = -INFINITY, l = 0.f;
             int n_local = 0;
+            // two-pass plans: this thread's row among all query rows of the plan, and the bias of the tile's node for it
+            const bool node_tiles = (STATS || BIAS) && item.seg == SEG_CTX;
+            const int64_t stat_row = node_tiles ? (static_cast<int64_t>(item.ctx_id) + (live ? tok : 0)) * p.H_q + item.kv_head * G + hg : 0;
+            float b_cur = 0.f, b_next = 0.f;
+            if (BIAS && node_tiles) b_next = p.bias[static_cast<int64_t>(item.first_tile.key_base) * p.stat_rows + stat_row];
 
             DevTile next_tile = item.first_tile;
             for (int t = item.tile_begin; t < item.tile_end; ++t) {
@@ -468,6 +496,12 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (t + 1 < item.tile_end) next_tile = p.tiles[t + 1];      // in flight while this tile is processed
                 if (!tile_visible(tile, g)) continue;
                 if (alt && (tcnt++ & 1u) != static_cast<uint32_t>(w)) continue;   // the other half's tile
+                if (BIAS) {
+                    // the next tile's record has had a whole tile to arrive: ask for its node's bias now, use it next time
+                    b_cur = b_next;
+                    if (node_tiles && t + 1 < item.tile_end)
+                        b_next = p.bias[static_cast<int64_t>(next_tile.key_base) * p.stat_rows + stat_row];
+                }
                 if (!__all_sync(0xffffffffu, mbar_wait(my_s_full, scnt & 1, &abort_flag, p.status))) { ok = false; break; }
                 ++scnt;
                 tc_fence_after();
@@ -477,6 +511,11 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     #pragma unroll
                     for (int c = 0; c < kTileN / 32; ++c) tmem_ld32(tS + c * 32, sr[c]);
                     tmem_ld_wait();
+                }
+                if (STATS) {                                           // S is in registers: the next product may overwrite it
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(my_p_full);
                 }
                 int limit = tile.n_valid;
                 if (tile.flags & TILE_CAUSAL) limit = min(limit, tok + g.off - tile.key_base + 1);
@@ -496,8 +535,12 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 #pragma unroll
                 for (int k = 0; k < 8; ++k) mxa[k] = fmaxf(mxa[k], s[kTileN - 8 + k]);
                 const float mx = fmaxf(max3(mxa[0], mxa[1], mxa[2]), fmaxf(max3(mxa[3], mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
-                const float m_new = fmaxf(m, mx * scale);
-                if (n_local == 0) {
+                const float m_new = fmaxf(m, BIAS ? mx * scale + b_cur : mx * scale);
+                if (STATS) {
+                    // no accumulator to keep consistent: the running sum simply follows the maximum
+                    l *= (m == -INFINITY) ? 0.f : fast_exp2(m - m_new);
+                    m = m_new;
+                } else if (n_local == 0) {
                     m = m_new;
                 } else {
                     const bool grow = m_new > m + kRescaleThreshold;
@@ -532,39 +575,58 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (!__all_sync(0xffffffffu, turn)) { ok = false; break; }
                 }
                 // p = 2^(s * scale - m): the multiply-subtract and the row sum run as packed two-float operations
-                const uint64_t scale2 = pack2(scale, scale), negm2 = pack2(-m_use, -m_use);
+                const uint64_t scale2 = pack2(scale, scale), negm2 = BIAS ? pack2(b_cur - m_use, b_cur - m_use) : pack2(-m_use, -m_use);
                 uint64_t sum2[2] = {0ull, 0ull};
                 // P is computed and published in quarters of 32 keys (16 packed registers): the PV product over a quarter
                 // runs while the next quarter's exponentials are computed, and only the last quarter's product plus the
                 // next S = Q K^T remain on this half's critical path.
                 #pragma unroll
                 for (int qq = 0; qq < 4; ++qq) {
-                    uint32_t pk[16];
-                    #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        float x0, x1;
-                        unpack2(fma2(pack2(s[qq * 32 + 2 * i], s[qq * 32 + 2 * i + 1]), scale2, negm2), x0, x1);
-                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-                        sum2[i & 1] = add2(sum2[i & 1], pack2(p0, p1));
-                        pk[i] = pack_bf16x2(p0, p1);
-                    }
-                    if (qq == 3 && !alt) {                                 // exponentials issued: the other half's turn
+                    if constexpr (STATS) {                                 // the sums only: nothing goes back to tensor memory
+                        #pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            float x0, x1;
+                            unpack2(fma2(pack2(s[qq * 32 + 2 * i], s[qq * 32 + 2 * i + 1]), scale2, negm2), x0, x1);
+                            sum2[i & 1] = add2(sum2[i & 1], pack2(fast_exp2(x0), fast_exp2(x1)));
+                        }
+                        if (qq == 3) {
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_tok + 8 * (1 - w));
+                        }
+                    } else {
+                        uint32_t pk[16];
+                        #pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            float x0, x1;
+                            unpack2(fma2(pack2(s[qq * 32 + 2 * i], s[qq * 32 + 2 * i + 1]), scale2, negm2), x0, x1);
+                            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                            sum2[i & 1] = add2(sum2[i & 1], pack2(p0, p1));
+                            pk[i] = pack_bf16x2(p0, p1);
+                        }
+                        if (qq == 3 && !alt) {                             // exponentials issued: the other half's turn
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_tok + 8 * (1 - w));
+                        }
+                        tmem_st16(tS + qq * 16, pk);
+                        tmem_st_wait();
+                        tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(bar_tok + 8 * (1 - w));
+                        if (lane == 0) mbar_arrive(my_p_full + 8 * qq);
                     }
-                    tmem_st16(tS + qq * 16, pk);
-                    tmem_st_wait();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(my_p_full + 8 * qq);
                 }
                 float sum[4];
                 unpack2(sum2[0], sum[0], sum[1]);
                 unpack2(sum2[1], sum[2], sum[3]);
                 l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
                 ++n_local;
+                if (STATS && (tile.flags & TILE_CTX_END)) {
+                    // the node's own tokens end here: its (maximum, sum) for this row, and a fresh start for the next node
+                    if (live) p.stats[static_cast<int64_t>(tile.key_base) * p.stat_rows + stat_row] = make_float2(m, l);
+                    m = -INFINITY; l = 0.f; n_local = 0;
+                }
             }
             if (!ok) break;
+            if (STATS) continue;                                        // no output in the statistics pass
 
             // ---- epilogue of the item -------------------------------------------------------------------------------
             if (n_local > 0) {
@@ -716,10 +778,10 @@ ape_attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
 }
 
-size_t attn_smem_bytes(int D, int q_bufs, int alt) {
+size_t attn_smem_bytes(int D, int mode) {
     const size_t tile = static_cast<size_t>(D / 64) * kSlabBytes;
     // Q halves + K stages + V stages
-    const int tiles = alt ? (1 + 3 + 3) : (q_bufs == 2) ? (4 + 2 + 1) : (2 + 2 + 2);
+    const int tiles = (mode == kAttnAlt) ? (1 + 3 + 3) : (mode == kAttnEncode) ? (4 + 2 + 1) : (2 + 2 + 2);
     return 1024 + tiles * tile + 512;
 }
 
@@ -742,24 +804,42 @@ static cudaError_t prepare_kernel(K kernel, int smem_bytes) {
     return e != cudaSuccess ? e : cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
 }
 
-cudaError_t attn_set_smem_attr(int D, int q_bufs, int alt, size_t smem_bytes) {
+template <int D>
+static cudaError_t prepare_mode(int mode, int n) {
+    switch (mode) {
+        case kAttnPrefill: return prepare_kernel(ape_attn_kernel<D, kAttnPrefill>, n);
+        case kAttnEncode:  return prepare_kernel(ape_attn_kernel<D, kAttnEncode>, n);
+        case kAttnAlt:     return prepare_kernel(ape_attn_kernel<D, kAttnAlt>, n);
+        case kAttnStats:   return prepare_kernel(ape_attn_kernel<D, kAttnStats>, n);
+        case kAttnBias:    return prepare_kernel(ape_attn_kernel<D, kAttnBias>, n);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t attn_set_smem_attr(int D, int mode, size_t smem_bytes) {
     const int n = static_cast<int>(smem_bytes);
-    if (alt) return D == 128 ? prepare_kernel(ape_attn_kernel<128, 1, true>, n) : prepare_kernel(ape_attn_kernel<64, 1, true>, n);
-    if (D == 128) return q_bufs == 2 ? prepare_kernel(ape_attn_kernel<128, 2, false>, n) : prepare_kernel(ape_attn_kernel<128, 1, false>, n);
-    return q_bufs == 2 ? prepare_kernel(ape_attn_kernel<64, 2, false>, n) : prepare_kernel(ape_attn_kernel<64, 1, false>, n);
+    return D == 128 ? prepare_mode<128>(mode, n) : prepare_mode<64>(mode, n);
+}
+
+template <int D>
+static void launch_mode(const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const CUtensorMap& tm_o,
+                        const SplitMaps& split, const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream) {
+    switch (p.mode) {
+        case kAttnPrefill: ape_attn_kernel<D, kAttnPrefill><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p); break;
+        case kAttnEncode:  ape_attn_kernel<D, kAttnEncode><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p); break;
+        case kAttnAlt:     ape_attn_kernel<D, kAttnAlt><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p); break;
+        case kAttnStats:   ape_attn_kernel<D, kAttnStats><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p); break;
+        case kAttnBias:    ape_attn_kernel<D, kAttnBias><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p); break;
+        default: break;
+    }
 }
 
 cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const CUtensorMap& tm_o,
                         const SplitMaps& split, const AttnParams& p, int n_cta, size_t smem_bytes, cudaStream_t stream)
 {
-    if (p.alt_halves) {
-        if (D == 128) ape_attn_kernel<128, 1, true><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
-        else ape_attn_kernel<64, 1, true><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
-    }
-    else if (D == 128 && p.n_q_bufs == 2) ape_attn_kernel<128, 2, false><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
-    else if (D == 128) ape_attn_kernel<128, 1, false><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
-    else if (p.n_q_bufs == 2) ape_attn_kernel<64, 2, false><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
-    else ape_attn_kernel<64, 1, false><<<n_cta, kThreads, smem_bytes, stream>>>(tm_q, tm_k, tm_v, tm_o, split, p);
+    if (p.mode < kAttnPrefill || p.mode > kAttnBias) return cudaErrorInvalidValue;
+    if (D == 128) launch_mode<128>(tm_q, tm_k, tm_v, tm_o, split, p, n_cta, smem_bytes, stream);
+    else launch_mode<64>(tm_q, tm_k, tm_v, tm_o, split, p, n_cta, smem_bytes, stream);
     return cudaGetLastError();
 }
 

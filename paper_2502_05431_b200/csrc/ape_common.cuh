@@ -18,9 +18,11 @@ struct DevTile {
     int32_t key_base;  // index of the tile's first key inside the query segment / context (causal, growing tiles)
     int32_t flags;     // TILE_CAUSAL: apply the causal rule; TILE_GROWS: n_valid follows the segment's current length
 };
-enum : int32_t { TILE_CAUSAL = 1, TILE_GROWS = 2, TILE_SPLIT = 4 };
+enum : int32_t { TILE_CAUSAL = 1, TILE_GROWS = 2, TILE_SPLIT = 4, TILE_CTX_END = 8 };
 // TILE_SPLIT (encode plans): the tile's first split_r rows are the tail of the shared prefix (from `tok`), the rest are the
 // first tokens of the item's context; key_base is -split_r, so the causal rule sees the prefix keys as "before the context".
+// TILE_CTX_END (two-pass plans): the last tile of a context node's own tokens; such plans keep the node's index in key_base
+// of their context tiles (which are not causal and need no key index).
 
 // A run of tiles of one segment for one (request, KV head, row block): yields one partial (m, l, O~).
 struct DevItem {

@@ -32,6 +32,13 @@ cudaError_t launch_decode(int D, const CUtensorMap& tm_k, const CUtensorMap& tm_
                           int n_cta, size_t smem_bytes, cudaStream_t stream);
 
 // Tensor-core attention kernel shared by query prefill and context encoding.
+enum : int32_t {
+    kAttnPrefill = 0,   // long items, one Q buffer, two stages each of K and V
+    kAttnEncode = 1,    // many short items with a row block each: two Q buffers, one V stage
+    kAttnAlt = 2,       // row blocks of 128 rows: both halves read the same rows and take alternate tiles (three K/V stages)
+    kAttnStats = 3,     // first pass of a plan with separately scaled context nodes: per row and node, (max, sum) of its own tokens
+    kAttnBias = 4       // second pass of such a plan: prefill with a per-row, per-node bias on the context logits
+};
 struct AttnParams {
     const DevTile* tiles;
     const DevItem* items;
@@ -46,18 +53,22 @@ struct AttnParams {
     int32_t G;
     int32_t H_q;
     int32_t n_sib;                   // sibling CTAs per group (row blocks that stream the same tiles together)
-    int32_t n_q_bufs;                // 1: long items (prefill); 2: many short items (encode), see the kernel
     int32_t q_rows_are_pool;         // encode: Q / O rows are pool tokens (row = context start + i)
     int32_t split_r;                 // rows of a TILE_SPLIT tile that come from the prefix (a multiple of 8; 0: no such tiles)
     int32_t o_via_tma;               // two-buffer plans whose items all have their own Q: full halves of O leave through shared
                                      // memory (the item's Q buffer) and a bulk tensor store described by tm_o
-    int32_t alt_halves;              // one-buffer plans whose row blocks have 128 rows: both halves read the same rows and take
-                                     // alternate tiles; a slot then holds two partials of 128 rows (half 0, half 1)
+    int32_t mode;                    // kAttnPrefill ... kAttnBias; kAttnAlt: a slot holds two partials of 128 rows (half 0, half 1)
+    // kAttnStats / kAttnBias: context tiles carry their node in key_base and TILE_CTX_END on a node's last tile; the value of
+    // node n for row (request row base + token) * H_q + head is at index n * stat_rows + row; an item's ctx_id is its
+    // request's row base
+    float2* stats;                   // kAttnStats writes (running maximum, sum) in base-2 units
+    const float* bias;               // kAttnBias reads the bias (base-2 units) of the node's tokens
+    int64_t stat_rows;
     int* status;
 };
 
-size_t attn_smem_bytes(int D, int q_bufs, int alt);
-cudaError_t attn_set_smem_attr(int D, int q_bufs, int alt, size_t smem_bytes);
+size_t attn_smem_bytes(int D, int mode);
+cudaError_t attn_set_smem_attr(int D, int mode, size_t smem_bytes);
 // K and V boxes of split_r rows (prefix part) and 128 - split_r rows (context part) for TILE_SPLIT tiles
 struct SplitMaps { CUtensorMap ka, kb, va, vb; };
 cudaError_t launch_attn(int D, const CUtensorMap& tm_q, const CUtensorMap& tm_k, const CUtensorMap& tm_v, const CUtensorMap& tm_o,
@@ -95,6 +106,29 @@ struct MergeParams {
     int32_t D;
 };
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
+
+// Between the two passes of a plan with separately scaled context nodes (per-context form: every context a marked
+// top-level node; context trees): from the (maximum, sum) of every node's own tokens to the bias of its tokens' logits.
+// Bottom-up, a node's log2 mass A_n combines its own tokens and its children (a marked child enters with S * A_c, Eq. 11,
+// an unmarked one with A_c); top-down, the bias of a node is the sum of (S - 1) * A_a over the marked nodes a on its
+// path to the root, itself included: with it, one plain softmax over all context keys gives every node's tokens the
+// weight the hierarchical formula gives them.  A node's parent has a smaller index than the node.
+struct NodeBiasParams {
+    const DevNode* nodes;            // all requests' nodes; pad != 0: the node has tokens of its own
+    const DevReq* reqs;              // pad: the request's row base (rows before it in the plan)
+    const int32_t* req_node0;        // [n_req + 1]: the nodes of request r are req_node0[r] .. req_node0[r + 1] - 1
+    int32_t n_req;
+    const float2* stats;             // [n_nodes][stat_rows] from the statistics pass (base-2 units)
+    float* mass;                     // [n_nodes][stat_rows] scratch: A_n
+    float* bias;                     // [n_nodes][stat_rows] out
+    int64_t stat_rows;
+    float S;
+    int32_t H_q;
+    int32_t max_rows;                // largest q_len * H_q of a request
+    int32_t max_nodes;               // most nodes of a request
+    size_t smem_limit;               // dynamic shared memory a CTA may ask for on this device
+};
+cudaError_t launch_node_bias(const NodeBiasParams& p, cudaStream_t stream);
 
 // Merge of the shards of a context-sharded attend: the context segments of all shards combine by the hierarchical softmax
 // identity, then Eq. 5's scaling factor and the merge with the non-context segment.

@@ -311,6 +311,118 @@ cudaError_t launch_shard_merge(const ShardMergeParams& p, cudaStream_t stream)
     return cudaGetLastError();
 }
 
+namespace {
+
+__device__ __forceinline__ float logaddexp2(float a, float b) {
+    const float m = fmaxf(a, b);
+    if (m == -INFINITY) return -INFINITY;
+    return m + log2f(exp2f(a - m) + exp2f(b - m));
+}
+
+// One thread per query row (token, head) of a request; consecutive threads hold consecutive rows, so every access to the
+// [node][row] arrays is coalesced.
+__global__ void __launch_bounds__(256)
+ape_node_bias_kernel(const NodeBiasParams p)
+{
+    const int r = blockIdx.y;
+    const DevReq rq = p.reqs[r];
+    const int64_t local = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (local >= static_cast<int64_t>(rq.q_len) * p.H_q) return;
+    const int64_t row = static_cast<int64_t>(rq.pad) * p.H_q + local;
+    const int n0 = p.req_node0[r], n1 = p.req_node0[r + 1];
+    for (int n = n0; n < n1; ++n) p.mass[static_cast<int64_t>(n) * p.stat_rows + row] = -INFINITY;
+    for (int n = n1 - 1; n >= n0; --n) {                     // children before parents
+        const DevNode nd = p.nodes[n];
+        float own = -INFINITY;
+        if (nd.pad) {
+            const float2 st = p.stats[static_cast<int64_t>(n) * p.stat_rows + row];
+            if (st.y > 0.f) own = st.x + log2f(st.y);
+        }
+        const float A = logaddexp2(own, p.mass[static_cast<int64_t>(n) * p.stat_rows + row]);
+        p.mass[static_cast<int64_t>(n) * p.stat_rows + row] = A;
+        if (nd.parent >= 0) {
+            float* up = p.mass + static_cast<int64_t>(nd.parent) * p.stat_rows + row;
+            *up = logaddexp2(*up, nd.scaled ? p.S * A : A);
+        }
+    }
+    for (int n = n0; n < n1; ++n) {                          // parents before children
+        const DevNode nd = p.nodes[n];
+        const float A = p.mass[static_cast<int64_t>(n) * p.stat_rows + row];
+        float b = (nd.parent >= 0) ? p.bias[static_cast<int64_t>(nd.parent) * p.stat_rows + row] : 0.f;
+        if (nd.scaled && A > -INFINITY) b += (p.S - 1.f) * A;
+        p.bias[static_cast<int64_t>(n) * p.stat_rows + row] = b;
+    }
+}
+
+// The same computation with a request's nodes x 32 rows in shared memory: a CTA takes 32 consecutive rows (lane = row).
+// Reading the statistics and writing the biases is spread over the eight warps (node n goes to warp n mod 8, 256
+// contiguous bytes per node); the two walks over the tree, which are sequential in the node index, are one warp's work
+// on shared memory instead of a chain of dependent global-memory accesses per node.
+constexpr int kBiasRows = 32;
+__global__ void __launch_bounds__(256)
+ape_node_bias_smem_kernel(const NodeBiasParams p)
+{
+    extern __shared__ float val[];                           // [nodes of the request][32]: own mass, then A_n, then the bias
+    const int r = blockIdx.y;
+    const DevReq rq = p.reqs[r];
+    const int64_t n_rows = static_cast<int64_t>(rq.q_len) * p.H_q;
+    const int64_t local = static_cast<int64_t>(blockIdx.x) * kBiasRows + (threadIdx.x & 31);
+    if (static_cast<int64_t>(blockIdx.x) * kBiasRows >= n_rows) return;
+    const bool live = local < n_rows;
+    const int64_t row = static_cast<int64_t>(rq.pad) * p.H_q + (live ? local : 0);
+    const int n0 = p.req_node0[r], n_nodes = p.req_node0[r + 1] - n0;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int i = warp; i < n_nodes; i += 8) {
+        float own = -INFINITY;
+        if (live && p.nodes[n0 + i].pad) {
+            const float2 st = p.stats[static_cast<int64_t>(n0 + i) * p.stat_rows + row];
+            if (st.y > 0.f) own = st.x + log2f(st.y);
+        }
+        val[i * kBiasRows + lane] = own;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        for (int i = n_nodes - 1; i >= 0; --i) {             // children before parents
+            const DevNode nd = p.nodes[n0 + i];
+            if (nd.parent >= 0) {
+                const float A = val[i * kBiasRows + lane];
+                float* up = &val[(nd.parent - n0) * kBiasRows + lane];
+                *up = logaddexp2(*up, nd.scaled ? p.S * A : A);
+            }
+        }
+        for (int i = 0; i < n_nodes; ++i) {                  // parents before children
+            const DevNode nd = p.nodes[n0 + i];
+            const float A = val[i * kBiasRows + lane];
+            float b = (nd.parent >= 0) ? val[(nd.parent - n0) * kBiasRows + lane] : 0.f;
+            if (nd.scaled && A > -INFINITY) b += (p.S - 1.f) * A;
+            val[i * kBiasRows + lane] = b;
+        }
+    }
+    __syncthreads();
+    if (live)
+        for (int i = warp; i < n_nodes; i += 8) p.bias[static_cast<int64_t>(n0 + i) * p.stat_rows + row] = val[i * kBiasRows + lane];
+}
+
+}  // namespace
+
+cudaError_t launch_node_bias(const NodeBiasParams& p, cudaStream_t stream)
+{
+    if (p.n_req <= 0 || p.max_rows <= 0) return cudaSuccess;
+    const size_t smem = static_cast<size_t>(p.max_nodes) * kBiasRows * sizeof(float);
+    if (p.max_nodes > 0 && smem <= p.smem_limit) {
+        if (smem > 48 * 1024 &&
+            cudaFuncSetAttribute(ape_node_bias_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+            return cudaGetLastError();
+        const dim3 grid(static_cast<unsigned>((p.max_rows + kBiasRows - 1) / kBiasRows), static_cast<unsigned>(p.n_req));
+        ape_node_bias_smem_kernel<<<grid, 256, smem, stream>>>(p);
+        return cudaGetLastError();
+    }
+    // too many nodes for shared memory: the per-node arrays stay in global memory
+    const dim3 grid(static_cast<unsigned>((p.max_rows + 255) / 256), static_cast<unsigned>(p.n_req));
+    ape_node_bias_kernel<<<grid, 256, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream)
 {
     const long long warps = static_cast<long long>(p.n_groups) * p.rows_per_slot;

@@ -14,7 +14,7 @@ LLAMA = dict(H_q=32, H_kv=8, d=128)
 
 def _check(b, mode, parents, scaled=None, kv_extra=0):
     out, lse, n = gpu_attend(b, mode, tree=(parents, scaled), kv_extra=kv_extra)
-    assert n == 2
+    assert n == (4 if mode == libape.APE_PREFILL else 2)      # prefill: statistics pass, biases, biased prefill, merge
     for r, rq in enumerate(b.requests):
         q, p, c, k = b.views(r)
         if kv_extra:
@@ -94,3 +94,18 @@ def test_malformed_trees_are_refused():
     with pytest.raises(libape.ApeError) as e:          # the sharded hand-out is defined for Eq. 5 only
         plan.attend_partial(0.9, ws, o, l, o.clone(), l.clone())
     assert e.value.code == -10
+
+
+def test_more_nodes_than_shared_memory_holds():
+    """1,900 one- to three-token contexts, every one a marked top-level node (Eq. 11-12): the walk over the nodes between the
+    two passes then keeps its per-node arrays in global memory instead of shared memory."""
+    import random
+    rnd = random.Random(5)
+    lens = [rnd.randint(1, 3) for _ in range(1900)]
+    b = wl.make_batch(H_q=8, H_kv=2, d=64, l_P=4, ctx_lens=[lens], l_q=9, seed=41, T=0.9, S=0.8, name="many_nodes")
+    out, lse, n = gpu_attend(b, libape.APE_PREFILL, per_context=True)
+    assert n == 4
+    q, p, c, k = b.views(0)
+    ref = orc.attend(q, p, c, k, b.T, b.S, per_context=True)
+    compare(out, ref.out.float(), "many nodes")
+    assert (lse.double() - ref.lse).abs().max().item() < 2e-3
