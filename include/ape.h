@@ -114,8 +114,11 @@ int ape_attend_plan(ape_handle_t handle, const ape_shape_t *shape, const ape_kv_
  * context C_i keeps its own softmax and enters the final merge with S * LogSumExp_i, i.e. the context mass is
  * sum_i Z_i^S instead of Eq. 5's (sum_i Z_i)^S.  The two forms agree when S = 1 or when there is one context; this
  * form depends on the context boundaries (contexts are never fused), and is the building block of the
- * tree-structured merge the paper names as a future direction.  Launch with ape_attend as usual.  Work items are
- * cut at every context boundary, so this form is slower when contexts are short.
+ * tree-structured merge the paper names as a future direction.  Launch with ape_attend as usual.
+ * APE_PREFILL plans run in two passes (ape_attend then launches four kernels): per query row the log-sum-exp of every
+ * context, then the same attention as ape_attend_plan with (S - 1) * LogSumExp_i added to the logits of context i, which
+ * gives its tokens exactly the weights of Eq. 11-12; the plan's workspace also holds 16 bytes per (context, query row,
+ * query head).  APE_DECODE plans keep one partial per context and cut their work items at every context boundary.
  */
 int ape_attend_plan_per_context(ape_handle_t handle, const ape_shape_t *shape, const ape_kv_pool_t *pool,
                                 const ape_rows_t *q, const ape_rows_t *out, float *lse,
@@ -135,7 +138,10 @@ int ape_attend_plan_per_context(ape_handle_t handle, const ape_shape_t *shape, c
  * family are printed formulas: one node per context gives Eq. 11-12 (ape_attend_plan_per_context), one tree over all
  * contexts gives Eq. 5 (ape_attend_plan).  The paper prints no formula for deeper hierarchies; where S applies along a
  * branch is this library's reading, made explicit by `scaled`.
- * Launch with ape_attend.  Work items are cut at node boundaries.  APE_ERR_INVALID_ARG for a malformed tree.
+ * Launch with ape_attend.  APE_PREFILL plans run in two passes like the per-context form (the bias of a node's tokens is
+ * the sum of (S - 1) * A_a over the scaled nodes a on its path to the top, itself included; 16 bytes of workspace per
+ * (node, query row, query head)); APE_DECODE plans cut their work items at node boundaries and merge the partials with a
+ * stack of accumulators.  APE_ERR_INVALID_ARG for a malformed tree.
  */
 int ape_attend_plan_tree(ape_handle_t handle, const ape_shape_t *shape, const ape_kv_pool_t *pool,
                          const ape_rows_t *q, const ape_rows_t *out, float *lse,
