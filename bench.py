@@ -65,9 +65,10 @@ def decode_bytes(n_req: int, tokens_per_req: int) -> float:
 # cached tokens).  Valid only for the kernel sources the counters were taken with: the figure is dropped (null) as
 # soon as the hash of those sources changes.
 NCU_TRAFFIC = {
-    "prefill": {"bytes": 2 * (266.98e6 + 11.47e6), "sources": ["ape_attn.cu", "ape_tcgen05.cuh", "ape_common.cuh"], "sha": "9d1b4479c5180aef"},
-    "decode": {"bytes": (1.05512e9 + 4.23e6) * (8409907200.0 / 1053835264.0), "sources": ["ape_decode.cu", "ape_common.cuh"], "sha": "3b704785906cb068"},
-    "rope": {"bytes": 2 * ((131.30e6 + 87.13e6) + (131.30e6 + 82.04e6) + (524.91e6 + 479.47e6)), "sources": ["ape_rope.cu"], "sha": "f5898872292cd437"},
+    "prefill": {"bytes": 2 * (267.04e6 + 11.59e6), "sources": ["ape_attn.cu", "ape_tcgen05.cuh", "ape_common.cuh"], "sha": "3ec78f118ba6054c"},
+    "encode": {"bytes": 2 * (792.07e6 + 485.03e6), "sources": ["ape_attn.cu", "ape_tcgen05.cuh", "ape_common.cuh"], "sha": "3ec78f118ba6054c"},
+    "decode": {"bytes": (1.05511e9 + 4.18e6) * (8409907200.0 / 1053835264.0), "sources": ["ape_decode.cu", "ape_common.cuh"], "sha": "350774570d2381af"},
+    "rope": {"bytes": 2 * ((131.30e6 + 86.35e6) + (131.30e6 + 82.34e6) + (524.94e6 + 479.29e6)), "sources": ["ape_rope.cu"], "sha": "eb5f0c0e67beef74"},
 }
 
 
@@ -595,7 +596,7 @@ def main():
     ridge = peaks["tf_burst"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
     enc["roofline"] = {"bound": "hbm" if fl_encode / enc_bytes < ridge else "tensor", "algorithmic_bytes": enc_bytes,
                        "flop_per_byte": fl_encode / enc_bytes, "ridge_flop_per_byte": ridge, "achieved": enc_gbs, "peak": peaks["hbm_gbs"],
-                       "unit": "GB/s", "frac": enc_gbs / peaks["hbm_gbs"], "traffic": None,
+                       "unit": "GB/s", "frac": enc_gbs / peaks["hbm_gbs"], "traffic": ncu_traffic("encode"),
                        "what": "Q read + O written once per row, K/V read once per context; the tensor fractions above are the other bound"}
     tf_prefill = pre["tflops"]
     gbs_decode = by_decode_total / (dec_total_ms * 1e-3) / 1e9

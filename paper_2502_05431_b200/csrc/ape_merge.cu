@@ -359,6 +359,11 @@ ape_node_bias_kernel(const NodeBiasParams p)
 // contiguous bytes per node); the two walks over the tree, which are sequential in the node index, are one warp's work
 // on shared memory instead of a chain of dependent global-memory accesses per node.
 constexpr int kBiasRows = 32;
+__device__ __forceinline__ float logaddexp2_fast(float a, float b) {
+    const float m = fmaxf(a, b);
+    if (m == -INFINITY) return -INFINITY;
+    return m + fast_log2(fast_exp2(a - m) + fast_exp2(b - m));
+}
 __global__ void __launch_bounds__(256)
 ape_node_bias_smem_kernel(const NodeBiasParams p)
 {
@@ -372,29 +377,35 @@ ape_node_bias_smem_kernel(const NodeBiasParams p)
     const int64_t row = static_cast<int64_t>(rq.pad) * p.H_q + (live ? local : 0);
     const int n0 = p.req_node0[r], n_nodes = p.req_node0[r + 1] - n0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the node records (parent, scaled) behind the values, so that the walks below read shared memory only
+    int2* rec = reinterpret_cast<int2*>(val + static_cast<size_t>(n_nodes) * kBiasRows);
+    for (int i = threadIdx.x; i < n_nodes; i += 256) {
+        const DevNode nd = p.nodes[n0 + i];
+        rec[i] = make_int2(nd.parent >= 0 ? nd.parent - n0 : -1, nd.scaled);
+    }
     for (int i = warp; i < n_nodes; i += 8) {
         float own = -INFINITY;
         if (live && p.nodes[n0 + i].pad) {
             const float2 st = p.stats[static_cast<int64_t>(n0 + i) * p.stat_rows + row];
-            if (st.y > 0.f) own = st.x + log2f(st.y);
+            if (st.y > 0.f) own = st.x + fast_log2(st.y);
         }
         val[i * kBiasRows + lane] = own;
     }
     __syncthreads();
     if (warp == 0) {
         for (int i = n_nodes - 1; i >= 0; --i) {             // children before parents
-            const DevNode nd = p.nodes[n0 + i];
-            if (nd.parent >= 0) {
+            const int2 nd = rec[i];
+            if (nd.x >= 0) {
                 const float A = val[i * kBiasRows + lane];
-                float* up = &val[(nd.parent - n0) * kBiasRows + lane];
-                *up = logaddexp2(*up, nd.scaled ? p.S * A : A);
+                float* up = &val[nd.x * kBiasRows + lane];
+                *up = logaddexp2_fast(*up, nd.y ? p.S * A : A);
             }
         }
         for (int i = 0; i < n_nodes; ++i) {                  // parents before children
-            const DevNode nd = p.nodes[n0 + i];
+            const int2 nd = rec[i];
             const float A = val[i * kBiasRows + lane];
-            float b = (nd.parent >= 0) ? val[(nd.parent - n0) * kBiasRows + lane] : 0.f;
-            if (nd.scaled && A > -INFINITY) b += (p.S - 1.f) * A;
+            float b = (nd.x >= 0) ? val[nd.x * kBiasRows + lane] : 0.f;
+            if (nd.y && A > -INFINITY) b += (p.S - 1.f) * A;
             val[i * kBiasRows + lane] = b;
         }
     }
@@ -408,7 +419,7 @@ ape_node_bias_smem_kernel(const NodeBiasParams p)
 cudaError_t launch_node_bias(const NodeBiasParams& p, cudaStream_t stream)
 {
     if (p.n_req <= 0 || p.max_rows <= 0) return cudaSuccess;
-    const size_t smem = static_cast<size_t>(p.max_nodes) * kBiasRows * sizeof(float);
+    const size_t smem = static_cast<size_t>(p.max_nodes) * (kBiasRows * sizeof(float) + sizeof(int2));
     if (p.max_nodes > 0 && smem <= p.smem_limit) {
         if (smem > 48 * 1024 &&
             cudaFuncSetAttribute(ape_node_bias_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
