@@ -377,19 +377,18 @@ ape_node_bias_smem_kernel(const NodeBiasParams p)
     const int64_t row = static_cast<int64_t>(rq.pad) * p.H_q + (live ? local : 0);
     const int n0 = p.req_node0[r], n_nodes = p.req_node0[r + 1] - n0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // the node records (parent, scaled) behind the values, so that the walks below read shared memory only
+    // the node records (parent; scaled | 2 * has tokens) behind the values, so that everything below reads shared memory only
     int2* rec = reinterpret_cast<int2*>(val + static_cast<size_t>(n_nodes) * kBiasRows);
     for (int i = threadIdx.x; i < n_nodes; i += 256) {
         const DevNode nd = p.nodes[n0 + i];
-        rec[i] = make_int2(nd.parent >= 0 ? nd.parent - n0 : -1, nd.scaled);
+        rec[i] = make_int2(nd.parent >= 0 ? nd.parent - n0 : -1, (nd.scaled ? 1 : 0) | (nd.pad ? 2 : 0));
     }
-    for (int i = warp; i < n_nodes; i += 8) {
-        float own = -INFINITY;
-        if (live && p.nodes[n0 + i].pad) {
-            const float2 st = p.stats[static_cast<int64_t>(n0 + i) * p.stat_rows + row];
-            if (st.y > 0.f) own = st.x + fast_log2(st.y);
-        }
-        val[i * kBiasRows + lane] = own;
+    __syncthreads();
+    #pragma unroll 4
+    for (int i = warp; i < n_nodes; i += 8) {                // independent loads: several in flight per warp
+        float2 st = make_float2(0.f, 0.f);
+        if (live && (rec[i].y & 2)) st = p.stats[static_cast<int64_t>(n0 + i) * p.stat_rows + row];
+        val[i * kBiasRows + lane] = (st.y > 0.f) ? st.x + fast_log2(st.y) : -INFINITY;
     }
     __syncthreads();
     if (warp == 0) {
@@ -398,14 +397,14 @@ ape_node_bias_smem_kernel(const NodeBiasParams p)
             if (nd.x >= 0) {
                 const float A = val[i * kBiasRows + lane];
                 float* up = &val[nd.x * kBiasRows + lane];
-                *up = logaddexp2_fast(*up, nd.y ? p.S * A : A);
+                *up = logaddexp2_fast(*up, (nd.y & 1) ? p.S * A : A);
             }
         }
         for (int i = 0; i < n_nodes; ++i) {                  // parents before children
             const int2 nd = rec[i];
             const float A = val[i * kBiasRows + lane];
             float b = (nd.x >= 0) ? val[nd.x * kBiasRows + lane] : 0.f;
-            if (nd.y && A > -INFINITY) b += (p.S - 1.f) * A;
+            if ((nd.y & 1) && A > -INFINITY) b += (p.S - 1.f) * A;
             val[i * kBiasRows + lane] = b;
         }
     }
