@@ -128,3 +128,24 @@ def test_shared_context_plan_under_a_budget():
     for r, rq in enumerate(b.requests):
         ref = oracle_attend(b, r, l_k=rq.query_kv[1] + 2)
         compare(out[r:r + 1], ref.out.float(), f"budget_shared req {r}")
+
+
+@pytest.mark.parametrize("budget", [5, 148])
+def test_two_pass_forms_under_another_split(budget):
+    """The per-context form in prefill (two passes: node statistics, biased prefill) with the context run cut into few and
+    into many items: a node's tiles never straddle two items, long nodes included (one context of 40 tiles), and the
+    result does not depend on where the cuts fall."""
+    from oracle import ape_oracle as orc
+    h = handle()
+    b = wl.make_batch(**LLAMA, l_P=20, ctx_lens=[[5000, 130, 1, 255, 700, 64, 64, 64]], l_q=70, l_k=90, seed=45, T=0.8, S=0.7,
+                      name="two_pass_split")
+    try:
+        h.set_sm_budget(budget)
+        out, lse, n = gpu_attend(b, libape.APE_PREFILL, per_context=True)
+    finally:
+        h.set_sm_budget(0)
+    assert n == 4
+    q, p, c, k = b.views(0)
+    ref = orc.attend(q, p, c, k, b.T, b.S, per_context=True)
+    compare(out, ref.out.float(), f"two-pass per-context, budget {budget}")
+    assert (lse.double() - ref.lse).abs().max().item() < 2e-3
