@@ -187,6 +187,17 @@ int ape_plan_destroy(ape_plan_t plan);
 int ape_attend(ape_plan_t plan, float T, float S, int64_t kv_extra,
                void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * The whole of Eq. 5 in one call, for callers who do not keep a plan: the arguments are the paper's statement of the
+ * problem (section "Formulation": the query rows, the shared prefix, the contexts, the query's own keys, T and S) in
+ * the layout of ape_attend_plan.  Plans, allocates the plan's scratch, launches on `stream`, waits for the stream,
+ * frees everything again.  Synchronous, and it pays the planning and two device allocations on every call: loops
+ * (a decode loop above all) should plan once and call ape_attend.  APE_DECODE here means kv_extra = 0.
+ */
+int ape_attend_once(ape_handle_t handle, const ape_shape_t *shape, const ape_kv_pool_t *pool,
+                    const ape_rows_t *q, const ape_rows_t *out, float *lse,
+                    const ape_request_t *requests, int32_t n_req, ape_mode_t mode, float T, float S, void *stream);
+
 /* Launch the context pre-encoding attention of an encode plan.  No T, no S (they apply to queries only).  An encode
  * plan writes its outputs directly and needs no scratch (ape_plan_workspace_bytes gives 0): `workspace` and
  * `workspace_bytes` are accepted so that all launches look alike, and are ignored (NULL / 0 are fine). */

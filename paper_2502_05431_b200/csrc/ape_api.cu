@@ -1088,6 +1088,23 @@ int ape_attend(ape_plan_t p, float T, float S, int64_t kv_extra, void* workspace
     return attend_impl(p, T, S, kv_extra, workspace, ws_bytes, stream_v, nullptr);
 }
 
+int ape_attend_once(ape_handle_t h, const ape_shape_t* shape, const ape_kv_pool_t* pool, const ape_rows_t* q,
+                    const ape_rows_t* out, float* lse, const ape_request_t* reqs, int32_t n_req, ape_mode_t mode, float T, float S,
+                    void* stream_v) {
+    ape_plan_t plan = nullptr;
+    int rc = ape_attend_plan(h, shape, pool, q, out, lse, reqs, n_req, mode, &plan);
+    if (rc) return rc;
+    DeviceGuard guard(h->device);
+    void* ws = nullptr;
+    if (!guard.ok) rc = APE_ERR_CUDA;
+    if (!rc && plan->ws_bytes > 0 && cudaMalloc(&ws, plan->ws_bytes) != cudaSuccess) { ws = nullptr; rc = APE_ERR_NOMEM; }
+    if (!rc) rc = ape_attend(plan, T, S, 0, ws, plan->ws_bytes, stream_v);
+    if (!rc && cudaStreamSynchronize(static_cast<cudaStream_t>(stream_v)) != cudaSuccess) rc = APE_ERR_CUDA;
+    if (ws) cudaFree(ws);
+    ape_plan_destroy(plan);
+    return rc;
+}
+
 int ape_attend_partial(ape_plan_t p, float T, int64_t kv_extra, void* workspace, size_t ws_bytes, const ape_partials_t* part,
                        void* stream_v) {
     if (!part) return APE_ERR_INVALID_ARG;

@@ -22,7 +22,7 @@ EXPORTS = ["ape_create", "ape_destroy", "ape_attend_plan", "ape_encode_plan", "a
            "ape_get_status", "ape_status_string", "ape_decode_noalloc", "ape_attend_plan_per_context",
            "ape_rope_runs_for_request", "ape_rope_plan", "ape_rope_write", "ape_attend_plan_shared",
            "ape_attend_partial", "ape_merge_shards", "ape_selftest_timeout", "ape_selftest_timeout_noalloc",
-           "ape_set_sm_budget", "ape_get_status_stream", "ape_decode_step_host", "ape_attend_plan_tree"]
+           "ape_set_sm_budget", "ape_get_status_stream", "ape_decode_step_host", "ape_attend_plan_tree", "ape_attend_once"]
 
 
 class ApeError(RuntimeError):
@@ -84,6 +84,7 @@ def load() -> C.CDLL:
                                         C.POINTER(ape_rows_t), vp, C.POINTER(ape_span_t), C.POINTER(ape_span_t), C.c_int32,
                                         C.POINTER(vp)]
         lib.ape_plan_workspace_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
+        lib.ape_attend_once.argtypes = lib.ape_attend_plan.argtypes[:9] + [C.c_float, C.c_float, vp]
         lib.ape_plan_destroy.argtypes = [vp]
         lib.ape_attend.argtypes = [vp, C.c_float, C.c_float, C.c_int64, vp, C.c_size_t, vp]
         lib.ape_encode_contexts.argtypes = [vp, vp, C.c_size_t, vp]
@@ -211,6 +212,24 @@ class Handle:
     def set_sm_budget(self, n_sm: int) -> None:
         """ape_set_sm_budget: later plans use at most n_sm thread blocks (0: the whole device)."""
         _check(load().ape_set_sm_budget(self._h, int(n_sm)), "ape_set_sm_budget")
+
+    def attend_once(self, *, H_q: int, H_kv: int, d: int, k_pool: torch.Tensor, v_pool: torch.Tensor, q: torch.Tensor,
+                    out: torch.Tensor, requests: Sequence, mode: int, T: float, S: float, lse: Optional[torch.Tensor] = None,
+                    softmax_scale: float = 0.0, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """ape_attend_once: plan, launch, wait and clean up in one call (same arguments as attend_plan, plus T and S)."""
+        shape = ape_shape_t(H_q, H_kv, d, softmax_scale)
+        pool, qr, orows = _pool(k_pool, v_pool), _rows(q), _rows(out)
+        n = len(requests)
+        arr = (ape_request_t * max(n, 1))()
+        keep = []
+        for i, r in enumerate(requests):
+            spans = (ape_span_t * max(len(r.ctx), 1))(*[ape_span_t(int(s), int(l)) for s, l in r.ctx])
+            keep.append(spans)
+            arr[i] = ape_request_t(int(r.q_start), int(r.q_len), ape_span_t(*map(int, r.prefix)), spans, len(r.ctx),
+                                   ape_span_t(*map(int, r.query_kv)), int(r.query_kv_capacity))
+        _check(load().ape_attend_once(self._h, C.byref(shape), C.byref(pool), C.byref(qr), C.byref(orows),
+                                      lse.data_ptr() if lse is not None else None, arr, n, int(mode), float(T), float(S),
+                                      _stream_ptr(stream)), "ape_attend_once")
 
     def attend_plan(self, *, H_q: int, H_kv: int, d: int, k_pool: torch.Tensor, v_pool: torch.Tensor,
                     q: torch.Tensor, out: torch.Tensor, requests: Sequence, mode: int,

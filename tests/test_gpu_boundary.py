@@ -149,3 +149,23 @@ def test_two_pass_forms_under_another_split(budget):
     ref = orc.attend(q, p, c, k, b.T, b.S, per_context=True)
     compare(out, ref.out.float(), f"two-pass per-context, budget {budget}")
     assert (lse.double() - ref.lse).abs().max().item() < 2e-3
+
+
+@pytest.mark.parametrize("mode", [libape.APE_PREFILL, libape.APE_DECODE])
+def test_attend_once_is_plan_launch_and_cleanup_in_one_call(mode):
+    l_q = 40 if mode == libape.APE_PREFILL else 1
+    b = wl.make_batch(**LLAMA, l_P=16, ctx_lens=[[64, 200, 130], [300]], l_q=l_q, l_k=l_q + 6, seed=46, T=0.8, S=0.9, name="once")
+    dev = torch.device("cuda:0")
+    q, k, v = b.q.to(dev), b.k_pool.to(dev), b.v_pool.to(dev)
+    out = torch.zeros_like(q)
+    lse = torch.zeros(q.shape[0], 32, dtype=torch.float32, device=dev)
+    handle().attend_once(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=q, out=out, requests=b.requests, mode=mode, T=b.T, S=b.S,
+                         lse=lse)
+    for r, rq in enumerate(b.requests):
+        ref = oracle_attend(b, r)
+        sl = slice(rq.q_start, rq.q_start + rq.q_len)
+        compare(out[sl].cpu(), ref.out.float(), f"attend_once req {r}")
+        assert (lse[sl].cpu().double() - ref.lse).abs().max().item() < 2e-3
+    with pytest.raises(libape.ApeError) as e:
+        handle().attend_once(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=q, out=out, requests=b.requests, mode=mode, T=-1.0, S=b.S)
+    assert e.value.code == -4          # APE_ERR_RANGE: nothing was launched, nothing is left allocated
