@@ -169,3 +169,45 @@ def test_attend_once_is_plan_launch_and_cleanup_in_one_call(mode):
     with pytest.raises(libape.ApeError) as e:
         handle().attend_once(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=q, out=out, requests=b.requests, mode=mode, T=-1.0, S=b.S)
     assert e.value.code == -4          # APE_ERR_RANGE: nothing was launched, nothing is left allocated
+
+
+def test_repeated_launches_give_the_same_bits():
+    """Every plan kind launched 25 times on the same workspace without a host synchronisation in between: the work split
+    and the merge order are fixed by the plan, so a run that differs from the first one in a single bit means a race
+    (a partial read before it was written, a stage recycled too early) -- the stand-in for a race detector here."""
+    dev = torch.device("cuda:0")
+    h = handle()
+
+    def stable(make_plan, launch, out):
+        plan = make_plan()
+        ws = plan.alloc_workspace() if plan.workspace_bytes else None
+        launch(plan, ws)
+        torch.cuda.synchronize()
+        first = out.clone()
+        assert not torch.isnan(first.float()).any()
+        for _ in range(25):
+            out.fill_(0)
+            launch(plan, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(out, first)
+        plan.close()
+        assert h.get_status() == 0
+
+    b = wl.make_batch(**LLAMA, l_P=64, ctx_lens=[[256] * 30, [700, 1, 300]], l_q=200, l_k=210, seed=47, T=0.9, S=0.8, name="stable",
+                      with_encode_q=True)
+    q, k, v = b.q.to(dev), b.k_pool.to(dev), b.v_pool.to(dev)
+    out = torch.zeros_like(q)
+    common = dict(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=q, out=out, requests=b.requests)
+    for kind in (dict(), dict(per_context=True), dict(tree=([[-1] + [0] * 29, [-1, 0, 0]], None))):
+        stable(lambda: h.attend_plan(mode=libape.APE_PREFILL, **common, **kind), lambda p, ws: p.attend(b.T, b.S, ws), out)
+    qe = b.q_enc.to(dev)
+    oe = torch.zeros_like(qe)
+    rq = b.requests[0]
+    stable(lambda: h.encode_plan(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=qe, out=oe, prefix=rq.prefix, ctx=rq.ctx),
+           lambda p, ws: p.encode_contexts(), oe[rq.ctx[0][0]:rq.ctx[-1][0] + rq.ctx[-1][1]])
+    d = wl.share_contexts(wl.make_batch(**LLAMA, l_P=16, ctx_lens=[[256] * 12] * 16, l_q=1, l_k=70, capacity=80, seed=48, T=0.9, S=0.9))
+    q, k, v = d.q.to(dev), d.k_pool.to(dev), d.v_pool.to(dev)
+    out = torch.zeros_like(q)
+    common = dict(H_q=32, H_kv=8, d=128, k_pool=k, v_pool=v, q=q, out=out, requests=d.requests, mode=libape.APE_DECODE)
+    for kind in (dict(), dict(shared=True)):
+        stable(lambda: h.attend_plan(**common, **kind), lambda p, ws: p.attend(d.T, d.S, ws, kv_extra=3), out)
