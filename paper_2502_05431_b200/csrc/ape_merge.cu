@@ -37,7 +37,9 @@ __device__ __forceinline__ void combine_segment(const float* __restrict__ ws_o, 
         for (int u = 0; u < kBatch; ++u) {
             const size_t slot = static_cast<size_t>(slot0) + static_cast<size_t>(i0 + u) * stride;
             const float* src = ws_o + (slot * rows_per_slot + row) * D + lane * VEC;
-            if (ml[u].y > 0.f) {                     // an empty partial's rows were never written
+            // Issued without waiting for (m, l): the row of an empty partial was never written, but it lies inside the
+            // workspace, and the fold below never looks at what was read from it.
+            if (i0 + u < n) {
                 if constexpr (VEC == 4) { const float4 t = *reinterpret_cast<const float4*>(src); x[u][0] = t.x; x[u][1] = t.y; x[u][2] = t.z; x[u][3] = t.w; }
                 else { const float2 t = *reinterpret_cast<const float2*>(src); x[u][0] = t.x; x[u][1] = t.y; }
             } else {
